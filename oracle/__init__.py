@@ -1,0 +1,37 @@
+"""CPU oracle for the partial-token GRPO policy-gradient step (NAT).
+
+TEST INFRASTRUCTURE ONLY.  This package is the slow, plain fp64 statement of
+what the CUDA library must compute.  It is imported by the tests, by the
+smoke check and by the benchmark's CPU-baseline leg; the product package never
+imports it and shares no code, table or constant generator with it.
+
+Parity status of each function (what pins it to something other than itself):
+
+  philox4x32_10     pinned: known-answer vectors of the published generator,
+                    and an independent big-integer restatement in the tests.
+  grpo_adv          pinned: z-score closed form for binary rewards, numpy
+                    mean/std cross-check, zero-sum invariant.
+  select            pinned: the paper's closed forms for the survival
+                    probabilities, E[L], exact enumeration of every cut value
+                    in rational arithmetic, binomial frequency test for URS.
+  compact           pinned: brute-force list comprehension, segment structure
+                    for prefix modes.
+  policy_loss_fwd   pinned: softmax rows sum to one, scipy log_softmax,
+                    old_logp == logp closed form, p = 1 full-token GRPO written
+                    as an independent double loop, exhaustive enumeration of
+                    masks / cuts (Proposition 1).
+  policy_loss_bwd   pinned: central finite differences of policy_loss_fwd,
+                    zero column sums, exhaustive enumeration of the gradient's
+                    expectation, saturated-clip zero gradient.
+"""
+from .philox import philox4x32_10  # noqa: F401
+from .nat_oracle import (  # noqa: F401
+    SEL_URS,
+    SEL_RPC,
+    SEL_DET,
+    grpo_adv,
+    select,
+    compact,
+    policy_loss_fwd,
+    policy_loss_bwd,
+)

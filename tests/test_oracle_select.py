@@ -1,0 +1,255 @@
+"""Pins for the oracle's RNG, advantages, selection and compaction (CPU only)."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import SEL_DET, SEL_RPC, SEL_URS, compact, grpo_adv, philox4x32_10, select
+from oracle.nat_oracle import urs_threshold
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ Philox
+def _kat():
+    rows = []
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            v = [int(x, 16) for x in line.split()]
+            rows.append((v[:4], v[4:6], v[6:]))
+    return rows
+
+
+def _philox_bigint(c, k):
+    """Independent restatement with Python integers (arbiter for both sides)."""
+    c = list(c)
+    k = list(k)
+    for r in range(10):
+        if r:
+            k = [(k[0] + 0x9E3779B9) % 2**32, (k[1] + 0xBB67AE85) % 2**32]
+        a = 0xD2511F53 * c[0]
+        b = 0xCD9E8D57 * c[2]
+        c = [(b >> 32) ^ c[1] ^ k[0], b % 2**32, (a >> 32) ^ c[3] ^ k[1], a % 2**32]
+    return c
+
+
+def test_philox_known_answers():
+    rows = _kat()
+    assert len(rows) == 3
+    for c, k, want in rows:
+        got = [int(x) for x in philox4x32_10(*c, *k)]
+        assert got == want
+        assert _philox_bigint(c, k) == want
+
+
+def test_philox_vectorised_matches_bigint():
+    rng = np.random.default_rng(5)
+    C = rng.integers(0, 2**32, size=(64, 4), dtype=np.uint64)
+    K = rng.integers(0, 2**32, size=(64, 2), dtype=np.uint64)
+    out = philox4x32_10(C[:, 0], C[:, 1], C[:, 2], C[:, 3], K[:, 0], K[:, 1])
+    for j in range(64):
+        want = _philox_bigint([int(x) for x in C[j]], [int(x) for x in K[j]])
+        assert [int(o[j]) for o in out] == want
+
+
+# --------------------------------------------------------------- advantages
+def test_adv_binary_closed_form():
+    # k ones among G: mu = k/G, sigma = sqrt(k (G-k)) / G   (Eq. grpo-adv)
+    G, eps = 8, 1e-6
+    for k in range(G + 1):
+        R = np.array([1.0] * k + [0.0] * (G - k), dtype=np.float32)
+        adv = grpo_adv(R, 1, G, eps)
+        sigma = math.sqrt(k * (G - k)) / G
+        hi = (1 - k / G) / (sigma + eps)
+        lo = (0 - k / G) / (sigma + eps)
+        want = np.array([hi] * k + [lo] * (G - k))
+        if k in (0, G):
+            assert np.all(adv == 0.0)
+        else:
+            np.testing.assert_allclose(adv, want, rtol=2e-7)
+
+
+def test_adv_matches_numpy_zscore_and_sums_to_zero():
+    rng = np.random.default_rng(1)
+    P, G, eps = 5, 6, 1e-6
+    R = rng.normal(size=P * G).astype(np.float32)
+    adv = grpo_adv(R, P, G, eps).reshape(P, G)
+    R2 = R.astype(np.float64).reshape(P, G)
+    want = (R2 - R2.mean(1, keepdims=True)) / (R2.std(1, ddof=0, keepdims=True) + eps)
+    np.testing.assert_allclose(adv, want, rtol=3e-7, atol=1e-7)
+    assert np.all(np.abs(adv.sum(1)) < 1e-5)
+    # groups are independent: changing one group leaves the others untouched
+    R3 = R.copy()
+    R3[:G] += 3.0
+    adv3 = grpo_adv(R3, P, G, eps).reshape(P, G)
+    assert np.array_equal(adv3[1:], adv[1:])
+
+
+# ---------------------------------------------------------------- selection
+def _cu(T):
+    return np.concatenate([[0], np.cumsum(T)]).astype(np.int32)
+
+
+def test_rpc_uniform_cutoff_closed_forms():
+    # q(l) = 1/T  =>  p_t = (T-t+1)/T,  sum_t p_t = (T+1)/2   (uniform cutoff)
+    T = np.array([1, 2, 7, 64, 1000])
+    mask, pi, cut = select(SEL_RPC, _cu(T), min_cut=1, seed=3)
+    cu = _cu(T)
+    for i, Ti in enumerate(T):
+        p = pi[cu[i]:cu[i + 1]]
+        t = np.arange(1, Ti + 1)
+        want = ((Ti - t + 1).astype(np.float32) / np.float32(Ti))
+        assert np.array_equal(p, want)
+        assert p[0] == 1.0 and np.all(np.diff(p) <= 0) and p[-1] > 0
+        assert abs(float(p.astype(np.float64).sum()) - (Ti + 1) / 2) < 1e-4 * Ti
+        assert 1 <= cut[i] <= Ti
+        assert np.array_equal(mask[cu[i]:cu[i + 1]], (t <= cut[i]).astype(np.uint8))
+
+
+def test_rpc_minimum_cutoff_closed_forms():
+    # p_t = 1 (t <= C), (T-t+1)/(T-C+1) (t > C); E[L] = (C+T)/2; 1/p bounded
+    C = 100
+    T = np.array([30, 100, 101, 250, 8192])
+    cu = _cu(T)
+    mask, pi, cut = select(SEL_RPC, cu, min_cut=C, seed=11, offset=5)
+    for i, Ti in enumerate(T):
+        Ci = min(C, Ti)
+        p = pi[cu[i]:cu[i + 1]].astype(np.float64)
+        t = np.arange(1, Ti + 1)
+        want = np.where(t <= Ci, 1.0, (Ti - t + 1) / (Ti - Ci + 1))
+        np.testing.assert_allclose(p, want, rtol=6e-8)
+        assert abs(p.sum() - (Ci + Ti) / 2) < 1e-4 * Ti
+        late = t > Ci      # the weight bound is stated for the positions past the mandatory prefix
+        assert np.all(1.0 / p[late] <= (Ti - Ci + 1) / (Ti - t[late] + 1) * (1 + 1e-6))
+        assert Ci <= cut[i] <= Ti
+    # a response shorter than C is kept whole with pi = 1
+    assert cut[0] == 30 and np.all(pi[:30] == 1.0) and np.all(mask[:30] == 1)
+
+
+def test_rpc_cut_law_exact_enumeration():
+    """Pr(L >= t) over every value of the 64-bit draw's quotient equals pi_t.
+
+    L = C + floor(u n / 2^64): the quotient takes each value j in {0..n-1} for
+    ceil((j+1) 2^64 / n) - ceil(j 2^64 / n) values of u, so the law is uniform
+    to within 2^-64 * n; rational arithmetic checks the survival function.
+    """
+    for T, C in [(9, 1), (40, 10), (13, 13)]:
+        n = T - C + 1
+        counts = [-((-(j + 1) * 2**64) // n) - (-((-j * 2**64) // n)) for j in range(n)]
+        assert sum(counts) == 2**64
+        _, pi, _ = select(SEL_RPC, _cu([T]), min_cut=C)
+        for t in range(1, T + 1):
+            surv = Fraction(sum(c for j, c in enumerate(counts) if C + j >= t), 2**64)
+            want = Fraction(1) if t <= C else Fraction(T - t + 1, n)
+            assert abs(surv - want) <= Fraction(n, 2**64)
+            assert abs(float(pi[t - 1]) - float(want)) <= 6e-8 * float(want)
+
+
+def test_rpc_cut_mean_over_seeds():
+    # E[L]/T = 1/2 + C/(2T)   (Appendix B.2)
+    T, C, S = 400, 100, 3000
+    cu = _cu([T] * 8)
+    cuts = np.concatenate([select(SEL_RPC, cu, min_cut=C, seed=s)[2] for s in range(S // 8)])
+    mean = cuts.mean() / T
+    want = 0.5 + C / (2 * T)
+    sd = math.sqrt(((T - C + 1) ** 2 - 1) / 12) / T / math.sqrt(len(cuts))
+    assert abs(mean - want) < 4 * sd
+    assert cuts.min() >= C and cuts.max() <= T
+    # distinct responses and distinct seeds give distinct draws
+    assert len(np.unique(cuts)) > 200
+
+
+def test_urs_threshold_and_pi():
+    assert urs_threshold(1.0) == 2**32
+    assert urs_threshold(0.5) == 2**31
+    assert urs_threshold(1e-12) == 1
+    with pytest.raises(ValueError):
+        urs_threshold(0.0)
+    T = np.array([5, 64, 333])
+    for p in (0.25, 0.5, 0.75):
+        mask, pi, cut = select(SEL_URS, _cu(T), p=p, seed=9)
+        assert cut is None
+        assert np.all(pi == np.float32(p))
+    mask, pi, _ = select(SEL_URS, _cu(T), p=1.0, seed=9)
+    assert np.all(mask == 1) and np.all(pi == 1.0)      # full-token case
+
+
+def test_urs_frequency_matches_p():
+    # E[m / pi] = 1 (Proposition 1): binomial z-test with fixed seeds
+    T = np.array([4096] * 16)
+    for p in (0.25, 0.5, 0.9):
+        mask, pi, _ = select(SEL_URS, _cu(T), p=p, seed=123, offset=7)
+        n = mask.size
+        z = (mask.sum() - n * p) / math.sqrt(n * p * (1 - p))
+        assert abs(z) < 4.0
+        est = (mask / pi.astype(np.float64)).mean()
+        assert abs(est - 1.0) < 4.0 * math.sqrt((1 - p) / p / n)
+
+
+def test_urs_keying():
+    """Draws depend on (seed, offset, response, position) and on nothing else."""
+    T = np.array([37, 64, 21])
+    cu = _cu(T)
+    base, _, _ = select(SEL_URS, cu, p=0.5, seed=42, offset=1)
+    # response 1 in isolation but with the same global index => same bits
+    k0, k1, off = 42, 0, 1
+    t0 = np.arange(64, dtype=np.uint64)
+    words = philox4x32_10(t0 >> np.uint64(2), 1, 0, off, k0, k1)
+    x = np.choose((t0 & np.uint64(3)).astype(np.int64), words)
+    assert np.array_equal(base[cu[1]:cu[2]], (x < 2**31).astype(np.uint8))
+    other_seed, _, _ = select(SEL_URS, cu, p=0.5, seed=43, offset=1)
+    other_off, _, _ = select(SEL_URS, cu, p=0.5, seed=42, offset=2)
+    hi_off, _, _ = select(SEL_URS, cu, p=0.5, seed=42, offset=1 + (1 << 32))
+    assert not np.array_equal(base, other_seed)
+    assert not np.array_equal(base, other_off)
+    assert not np.array_equal(base, hi_off)
+    # the prefix of a longer response equals the shorter response's draws
+    longer, _, _ = select(SEL_URS, _cu([50, 64, 21]), p=0.5, seed=42, offset=1)
+    assert np.array_equal(longer[:37], base[:37])
+
+
+def test_det_truncation():
+    T = np.array([1, 2, 9, 100])
+    cu = _cu(T)
+    mask, pi, cut = select(SEL_DET, cu, beta=0.5)
+    assert list(cut) == [1, 1, 4, 50]
+    assert np.all(pi == 1.0)
+    for i in range(len(T)):
+        assert mask[cu[i]:cu[i + 1]].sum() == cut[i]
+        assert np.all(mask[cu[i]:cu[i] + cut[i]] == 1)
+
+
+def test_empty_responses():
+    cu = _cu([0, 5, 0, 3, 0])
+    for mode in (SEL_URS, SEL_RPC, SEL_DET):
+        mask, pi, cut = select(mode, cu, p=0.5, min_cut=2, beta=0.5, seed=1)
+        assert mask.shape == (8,)
+        if cut is not None:
+            assert cut[0] == 0 and cut[2] == 0 and cut[4] == 0
+        si, sr, so, n = compact(mask, cu)
+        assert n == int(mask.sum()) and so[0] == 0 and so[1] == 0 and so[-1] == n
+
+
+# --------------------------------------------------------------- compaction
+def test_compact_brute_force_and_segments():
+    rng = np.random.default_rng(2)
+    T = rng.integers(1, 50, size=12)
+    cu = _cu(T)
+    mask = (rng.random(cu[-1]) < 0.4).astype(np.uint8)
+    si, sr, so, n = compact(mask, cu)
+    assert n == mask.sum()
+    assert np.array_equal(si, np.nonzero(mask)[0])
+    resp_of = np.repeat(np.arange(len(T)), T)
+    assert np.array_equal(sr, resp_of[si])
+    for i in range(len(T)):
+        assert so[i + 1] - so[i] == mask[cu[i]:cu[i + 1]].sum()
+    # prefix modes: the kept tokens of response i are [cu_i, cu_i + L_i)
+    mask, _, cut = select(SEL_RPC, cu, min_cut=3, seed=4)
+    si, sr, so, n = compact(mask, cu)
+    want = np.concatenate([np.arange(cu[i], cu[i] + cut[i]) for i in range(len(T))])
+    assert np.array_equal(si, want)
+    assert n == cut.sum()
