@@ -1,0 +1,188 @@
+/*
+ * nat.h - C ABI of the partial-token GRPO policy-gradient step (NAT, "Not All
+ * Tokens are Needed") for NVIDIA B200 (sm_100a).
+ *
+ * Notation (the paper's): P prompts, G responses per prompt, B = P*G
+ * responses; response i has length T_i and belongs to prompt i / G; the
+ * responses are packed back to back, cu_seqlens[i] is the index of the first
+ * token of response i and cu_seqlens[B] = N_tot.  Token n of the packed
+ * stream sits at 1-based position t = n - cu_seqlens[resp(n)] + 1.
+ * m is the selection mask, pi the inclusion probability, L_i the RPC cut,
+ * A_i the group-relative advantage, d the hidden size, V the vocabulary.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers owned by the caller unless the comment says
+ *     "host".  Nothing is retained after the call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work on it and return without synchronising.
+ *   - The library allocates no device memory: kernels that need scratch take
+ *     a caller-provided `workspace` whose size the matching *_workspace_bytes
+ *     function returns.  The workspace must be 256-byte aligned.
+ *   - Return value: NAT_OK, or a negative nat_status; on error nothing was
+ *     enqueued.  nat_last_error() gives a thread-local message.
+ *   - Device-side conditions that cannot be known at launch (a bounded wait
+ *     that ran out, n_sel above the stated capacity) are recorded in the
+ *     32-bit status word at the start of the workspace (see
+ *     NAT_DEV_* bits); kernels never trap.
+ */
+#ifndef NAT_H_
+#define NAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  NAT_OK = 0,
+  NAT_ERR_INVALID_ARG = -1, /* null pointer, negative size, p outside (0,1], ... */
+  NAT_ERR_UNSUPPORTED = -2, /* dtype/shape the kernels do not cover, wrong GPU architecture */
+  NAT_ERR_CAPACITY = -3,    /* workspace or output capacity too small */
+  NAT_ERR_CUDA = -4         /* a CUDA runtime/driver call failed; see nat_last_error() */
+} nat_status;
+
+/* Bits of the device status word (first 4 bytes of a loss workspace). */
+#define NAT_DEV_TIMEOUT 1u  /* a bounded mbarrier wait gave up; outputs are invalid */
+#define NAT_DEV_CAPACITY 2u /* *n_sel exceeded n_sel_cap; surplus rows were ignored */
+
+const char* nat_status_string(int status);
+const char* nat_last_error(void); /* host string, valid until the thread's next failing call */
+int nat_version(void);
+
+/* ---------------------------------------------------------------------------
+ * Group-relative advantage (Eq. grpo-adv, Section 2.2):
+ *   A_i = (R_i - mu) / (sigma + eps), mu and sigma the population mean and
+ *   standard deviation (1/G) of the G rewards of response i's prompt.
+ * rewards, adv: float32 [P*G].  Arithmetic is double in index order and the
+ * result is rounded once to float32, so it is reproducible bit for bit.
+ * A group with equal rewards gets A = 0.
+ * ------------------------------------------------------------------------- */
+int nat_grpo_adv(int32_t P, int32_t G, const float* rewards, float eps, float* adv, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Token selection (Section 3.1 "Random masking", URS; Section 4 RPC with the
+ * uniform and minimum-cutoff laws; deterministic truncation as the biased
+ * comparison).  Random draws are Philox4x32-10 outputs, a pure function of
+ * (seed, offset, response index, position):
+ *   key     = (seed_lo, seed_hi ^ offset_hi)
+ *   URS     token t uses word (t-1)%4 of counter ((t-1)/4, i, 0, offset_lo);
+ *           m = [x < thr], thr = clamp(floor(p 2^32), 1, 2^32), pi = thr/2^32.
+ *   RPC     response i draws counter (0, i, 1, offset_lo), u = x1 2^32 + x0,
+ *           C_i = min(max(min_cut,1), T_i), n = T_i - C_i + 1,
+ *           L_i = C_i + floor(u n / 2^64); m_t = [t <= L_i];
+ *           pi_t = 1 (t <= C_i), (T_i-t+1)/(T_i-C_i+1) otherwise (one float32
+ *           division, Eq. rpc-survival under the uniform law).
+ *   DET     K_i = max(1, floor(beta T_i)); m_t = [t <= K_i]; pi_t = 1.
+ * Outputs: mask uint8 [n_tot] (0/1), pi float32 [n_tot], cut_len int32 [B]
+ * (L_i or K_i, 0 for an empty response; may be NULL for URS, which leaves it
+ * untouched).  cu_seqlens int32 [B+1] on the device; n_tot is the host's copy
+ * of cu_seqlens[B].  T_i = 0 is allowed.
+ * Errors: NAT_ERR_INVALID_ARG for p outside (0,1], beta outside (0,1],
+ * min_cut < 0, B < 0, n_tot < 0 or null pointers.
+ * ------------------------------------------------------------------------- */
+typedef enum { NAT_SEL_URS = 0, NAT_SEL_RPC = 1, NAT_SEL_DET = 2 } nat_sel_mode;
+
+typedef struct {
+  int32_t mode;    /* nat_sel_mode */
+  int32_t min_cut; /* RPC: C (0 and 1 both mean the plain uniform cutoff) */
+  double p;        /* URS: inclusion probability in (0,1] */
+  double beta;     /* DET: kept fraction in (0,1] */
+  uint64_t seed;
+  uint64_t offset; /* caller's step counter: a new offset gives fresh draws */
+} nat_select_params;
+
+int nat_select(const nat_select_params* params /* host */, int32_t B, const int32_t* cu_seqlens,
+               int64_t n_tot, uint8_t* mask, float* pi, int32_t* cut_len, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Compaction of the selected tokens ("only included tokens contribute to
+ * backpropagation", Section 1; Eq. ht-estimator sums over m = 1 only).
+ *   sel_idx  int32 [cap]   ascending packed indices n with mask[n] != 0
+ *   sel_resp int32 [cap]   resp(sel_idx[k])
+ *   sel_offsets int32 [B+1] number of selected tokens in responses < i
+ *   n_sel    int32 device scalar = sel_offsets[B]
+ * cap is the number of elements the two lists can hold; if more tokens are
+ * selected the surplus is not written and *n_sel still reports the true count.
+ * workspace: nat_compact_workspace_bytes(n_tot) bytes.
+ * ------------------------------------------------------------------------- */
+size_t nat_compact_workspace_bytes(int64_t n_tot);
+int nat_compact(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8_t* mask,
+                int32_t* sel_idx, int32_t* sel_resp, int32_t* sel_offsets, int32_t* n_sel,
+                int64_t cap, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Policy loss over the selected tokens (ratio Eq. ratio, clipped surrogate
+ * Eq. grpo-surrogate, sequence/group mean Eq. grpo-obj, Horvitz-Thompson
+ * weights Eq. ht-estimator and Eq. rpc-ht; KL coefficient 0 as in the paper's
+ * experiments).  For selected token k (packed index n = sel_idx[k],
+ * response i = sel_resp[k], hidden row h):
+ *   z = W h (V logits, fp32 accumulation), lse = log sum_v exp z_v,
+ *   logp = z[targets[n]] - lse,  r = exp(logp - old_logp[n]),
+ *   S = min(r A_i, clip(r, 1-clip_lo, 1+clip_hi) A_i),
+ *   w = 1 / (pi[n] T_i B),   loss = - sum_k w S.
+ * The logits are never written to memory.
+ *
+ * dtype NAT_BF16: hidden, W, dHidden are bfloat16 and the projection runs on
+ * the tensor cores; requires d % 64 == 0.  dtype NAT_F32: float32 operands,
+ * plain fp32 arithmetic, any d and V (meant for small problems).
+ * hidden is [n_tot, d] row-major (row sel_idx[k] is used) or, with
+ * hidden_is_compact, [>= n_sel, d] with row k belonging to sel_idx[k].
+ * W is [V, d] row-major.  targets int32 [n_tot] in [0, V); old_logp, pi
+ * float32 [n_tot]; adv float32 [B].  n_sel is the device scalar written by
+ * nat_compact; n_sel_cap is a host upper bound on it (grid and workspace are
+ * sized from it; rows beyond it are ignored and NAT_DEV_CAPACITY is raised).
+ * Outputs: loss float32 device scalar; logp, lse float32 [n_sel_cap] (entries
+ * k < n_sel are written).  The reduction order is fixed, so the loss is
+ * reproducible run to run.
+ * workspace: nat_policy_loss_workspace_bytes(params, n_sel_cap); it is shared
+ * by forward and backward and holds nothing that must survive between them.
+ * ------------------------------------------------------------------------- */
+#define NAT_F32 0
+#define NAT_BF16 1
+
+typedef struct {
+  int32_t d;
+  int32_t V;
+  int32_t dtype; /* NAT_F32 | NAT_BF16 */
+  int32_t B;     /* number of responses (the batch mean's divisor) */
+  float clip_lo; /* ratio is clipped to [1-clip_lo, 1+clip_hi] */
+  float clip_hi;
+  int32_t hidden_is_compact;
+  int32_t accumulate_dW; /* backward: 0 overwrite dW, 1 add to it */
+} nat_loss_params;
+
+size_t nat_policy_loss_workspace_bytes(const nat_loss_params* params /* host */,
+                                       int64_t n_sel_cap);
+
+int nat_policy_loss_fwd(const nat_loss_params* params /* host */, const void* hidden,
+                        const void* W, const int32_t* targets, const float* old_logp,
+                        const float* adv, const float* pi, const int32_t* cu_seqlens,
+                        const int32_t* sel_idx, const int32_t* sel_resp, const int32_t* n_sel,
+                        int64_t n_sel_cap, float* loss, float* logp, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Backward of the loss above (the gradient of Eq. ht-estimator, Appendix A).
+ * With g_k = -dloss w A r 1[surrogate not saturated] (saturated: A > 0 and
+ * r > 1+clip_hi, or A < 0 and r < 1-clip_lo; A = 0 gives 0):
+ *   dz[k, v] = g_k (1[v = y_k] - exp(z_v - lse_k))      (z recomputed)
+ *   dHidden[k, :] = sum_v dz[k, v] W[v, :]     compact: row k <-> sel_idx[k]
+ *   dW[v, :]      = sum_k dz[k, v] h_k          float32 [V, d]
+ * logp and lse are the forward's outputs.  dloss is a device float scalar
+ * (NULL means 1).  dHidden has hidden's dtype, [n_sel_cap, d]; rows >= n_sel
+ * are not written.  With accumulate_dW the product is added to dW's contents.
+ * ------------------------------------------------------------------------- */
+int nat_policy_loss_bwd(const nat_loss_params* params /* host */, const void* hidden,
+                        const void* W, const int32_t* targets, const float* old_logp,
+                        const float* adv, const float* pi, const int32_t* cu_seqlens,
+                        const int32_t* sel_idx, const int32_t* sel_resp, const int32_t* n_sel,
+                        int64_t n_sel_cap, const float* logp, const float* lse,
+                        const float* dloss, void* dHidden, float* dW, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NAT_H_ */

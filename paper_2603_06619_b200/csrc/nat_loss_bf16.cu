@@ -1,0 +1,728 @@
+// bf16 policy loss on the Blackwell tensor cores (tcgen05 + TMEM + TMA).
+//
+// One warp-specialised persistent kernel template serves the four dense
+// contractions of the path; they differ in operand layout and epilogue:
+//
+//   kFwd  S = Hc W^T  (rows x V, K = d)  epilogue: online max / sum-exp and
+//                                        target-logit pick per row; the logits
+//                                        stay in tensor memory and registers.
+//   kDz   S = Hc W^T  recomputed         epilogue: -g exp(S - lse) -> bf16 into
+//                                        the bounded scratch dZ[chunk, V].
+//   kDh   dH = dZ W   (rows x d, K = V)  epilogue: + g W[y] (one-hot term) -> bf16.
+//   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 read-modify-write.
+//
+// Roles per CTA (192 threads): warp 0 issues TMA loads into a 4-stage shared
+// memory ring, warp 1 issues tcgen05.mma into one of two 128x256 fp32
+// accumulators in tensor memory, warps 2..5 drain the other accumulator.
+// Every mbarrier wait is bounded; a wait that runs out raises the block's
+// abort flag and NAT_DEV_TIMEOUT in the workspace's status word.
+#include <cuda_bf16.h>
+
+#include "nat_tc.cuh"
+#include "nat_token.cuh"
+
+namespace nat {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;               // 16 KB
+constexpr int kBBytes = BN * BK * 2;               // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;     // 48 KB
+constexpr int kBoxBytes = 64 * 64 * 2;             // one 64x64 box of an MN-major operand
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;                     // two 256-column accumulators
+constexpr int kGroupRows = 16;                     // row blocks that share a vocabulary sweep
+constexpr int kTilesPerSplit = 16;                 // vocabulary tiles per work unit
+constexpr int kChunkRows = 8192;                   // rows of the dZ scratch
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+
+enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3 };
+
+struct TcParams {
+  const int32_t* n_sel;
+  int cap;
+  int row0;        // first compact row handled by this launch
+  int chunk_rows;  // rows this launch may cover (multiple of 128)
+  int d, V;
+  int n_splits;    // vocabulary splits (kFwd, kDz)
+  int cap_pad;     // stride of the per-split partials
+  const int32_t* targets;
+  const int32_t* sel_idx;
+  float* part_m;
+  float* part_s;
+  float* zt;
+  const float* g;
+  const float* lse;
+  __nv_bfloat16* dZ;
+  int ldz;         // elements per dZ row
+  const __nv_bfloat16* W;
+  __nv_bfloat16* dH;
+  float* dW;
+  uint32_t* status;
+};
+
+struct Unit {
+  int mb;      // block along the accumulator's M dimension
+  int nt_lo;   // first and one-past-last block along N
+  int nt_hi;
+  int sp;      // vocabulary split (kFwd, kDz)
+};
+
+struct Shape {
+  int rows;     // valid rows of this launch
+  int n_units;
+  int kb;       // k-blocks per tile
+  int mblocks;
+  int nblocks;  // N blocks (kDh, kDw) or vocabulary tiles (kFwd, kDz)
+};
+
+template <int MODE>
+__device__ __forceinline__ Shape make_shape(const TcParams& p) {
+  Shape s;
+  int n = *p.n_sel;
+  n = n < p.cap ? n : p.cap;
+  int rows = n - p.row0;
+  rows = rows < 0 ? 0 : (rows > p.chunk_rows ? p.chunk_rows : rows);
+  s.rows = rows;
+  if (MODE == kFwd || MODE == kDz) {
+    s.mblocks = (rows + BM - 1) / BM;
+    s.nblocks = (p.V + BN - 1) / BN;
+    s.n_units = s.mblocks * p.n_splits;
+    s.kb = p.d / BK;
+  } else if (MODE == kDh) {
+    s.mblocks = (rows + BM - 1) / BM;
+    s.nblocks = (p.d + BN - 1) / BN;
+    s.n_units = s.mblocks * s.nblocks;
+    s.kb = (p.V + BK - 1) / BK;
+  } else {
+    s.mblocks = (p.V + BM - 1) / BM;
+    s.nblocks = (p.d + BN - 1) / BN;
+    s.kb = (rows + BK - 1) / BK;
+    s.n_units = rows > 0 ? s.mblocks * s.nblocks : 0;
+  }
+  return s;
+}
+
+// Units are ordered so that CTAs running side by side share operands in L2:
+// kFwd/kDz take groups of kGroupRows row blocks and, inside a group, walk the
+// vocabulary splits with the row block varying fastest.
+template <int MODE>
+__device__ __forceinline__ Unit decode_unit(const TcParams& p, const Shape& s, int u) {
+  Unit w;
+  if (MODE == kFwd || MODE == kDz) {
+    const int per_group = kGroupRows * p.n_splits;
+    const int grp = u / per_group;
+    const int rem = u - grp * per_group;
+    int rows_in_group = s.mblocks - grp * kGroupRows;
+    rows_in_group = rows_in_group < kGroupRows ? rows_in_group : kGroupRows;
+    w.sp = rem / rows_in_group;
+    w.mb = grp * kGroupRows + (rem - w.sp * rows_in_group);
+    w.nt_lo = (int)(((long long)w.sp * s.nblocks) / p.n_splits);
+    w.nt_hi = (int)(((long long)(w.sp + 1) * s.nblocks) / p.n_splits);
+  } else {
+    w.sp = 0;
+    w.mb = u / s.nblocks;
+    w.nt_lo = u - w.mb * s.nblocks;
+    w.nt_hi = w.nt_lo + 1;
+  }
+  return w;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1)
+nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+              const TcParams p) {
+  constexpr bool kAmn = (MODE == kDw);
+  constexpr bool kBmn = (MODE == kDh || MODE == kDw);
+  constexpr uint32_t kIdesc = tc::instr_desc_bf16(BM, BN, kAmn ? 1 : 0, kBmn ? 1 : 0);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);
+  uint64_t* full_bar = bars;                    // [kStages]
+  uint64_t* empty_bar = bars + kStages;         // [kStages]
+  uint64_t* tfull_bar = bars + 2 * kStages;     // [2]
+  uint64_t* tempty_bar = bars + 2 * kStages + 2;  // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      tc::mbar_init(&full_bar[s], 1);
+      tc::mbar_init(&empty_bar[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      tc::mbar_init(&tfull_bar[a], 1);
+      tc::mbar_init(&tempty_bar[a], 4);
+    }
+    *abort_flag = 0u;
+    tc::fence_barrier_init();
+    tc::fence_proxy_async();
+    tc::prefetch_tensormap(&mapA);
+    tc::prefetch_tensormap(&mapB);
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(tmem_slot, kTmemCols);
+    tc::tmem_relinquish();
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const Shape shape = make_shape<MODE>(p);
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < shape.n_units; u += gridDim.x) {
+        const Unit w = decode_unit<MODE>(p, shape, u);
+        for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt) {
+          for (int kb = 0; kb < shape.kb; ++kb, ++it) {
+            const int s = it % kStages;
+            const uint32_t ph = (it / kStages) & 1u;
+            if (!tc::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+            uint8_t* a_dst = smem + (size_t)s * kStageBytes;
+            uint8_t* b_dst = a_dst + kABytes;
+            tc::mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
+            if (MODE == kFwd || MODE == kDz) {
+              tc::tma_load_2d(a_dst, &mapA, &full_bar[s], kb * BK, p.row0 + w.mb * BM);
+              tc::tma_load_2d(b_dst, &mapB, &full_bar[s], kb * BK, nt * BN);
+            } else if (MODE == kDh) {
+              tc::tma_load_2d(a_dst, &mapA, &full_bar[s], kb * BK, w.mb * BM);
+#pragma unroll
+              for (int j = 0; j < BN / 64; ++j)
+                tc::tma_load_2d(b_dst + j * kBoxBytes, &mapB, &full_bar[s], nt * BN + j * 64,
+                                kb * BK);
+            } else {
+#pragma unroll
+              for (int j = 0; j < BM / 64; ++j)
+                tc::tma_load_2d(a_dst + j * kBoxBytes, &mapA, &full_bar[s], w.mb * BM + j * 64,
+                                kb * BK);
+#pragma unroll
+              for (int j = 0; j < BN / 64; ++j)
+                tc::tma_load_2d(b_dst + j * kBoxBytes, &mapB, &full_bar[s], nt * BN + j * 64,
+                                p.row0 + kb * BK);
+            }
+          }
+        }
+      }
+      if (!ok) {
+        // Loads already issued still complete on their own; give them a
+        // bounded chance to land before the block's shared memory is released.
+        const uint32_t pending = it < (uint32_t)kStages ? it : (uint32_t)kStages;
+        for (uint32_t j = 0; j < pending; ++j) {
+          const uint32_t jt = it - 1 - j;
+          const uint64_t t0 = tc::global_timer_ns();
+          while (!tc::mbar_try_wait(&full_bar[jt % kStages], (jt / kStages) & 1u)) {
+            if (tc::global_timer_ns() - t0 > 100000000ull) break;
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < shape.n_units; u += gridDim.x) {
+        const Unit w = decode_unit<MODE>(p, shape, u);
+        for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt, ++tcount) {
+          const uint32_t acc = tcount & 1u;
+          const uint32_t aph = (tcount >> 1) & 1u;
+          if (!tc::mbar_wait(&tempty_bar[acc], aph ^ 1u, abort_flag)) { ok = false; break; }
+          tc::fence_after_sync();
+          const uint32_t d_tmem = tmem_base + acc * BN;
+          for (int kb = 0; kb < shape.kb; ++kb, ++it) {
+            const int s = it % kStages;
+            const uint32_t ph = (it / kStages) & 1u;
+            if (!tc::mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
+            tc::fence_after_sync();
+            const uint32_t a_base = tc::smem_u32(smem + (size_t)s * kStageBytes);
+            const uint32_t b_base = a_base + kABytes;
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk) {
+              // K-major: 16 elements of K are 32 bytes inside the swizzled
+              // 128-byte row; 8-row groups are 1024 bytes apart.
+              // MN-major: 16 rows of K are two 8-row groups 1024 bytes apart
+              // (stride offset); 64-element groups along M/N are whole boxes
+              // apart (leading offset).
+              const uint64_t adesc =
+                  kAmn ? tc::smem_desc_sw128(a_base + kk * 2048, kBoxBytes, 1024)
+                       : tc::smem_desc_sw128(a_base + kk * 32, 16, 1024);
+              const uint64_t bdesc =
+                  kBmn ? tc::smem_desc_sw128(b_base + kk * 2048, kBoxBytes, 1024)
+                       : tc::smem_desc_sw128(b_base + kk * 32, 16, 1024);
+              tc::umma_bf16(d_tmem, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+            }
+            tc::umma_commit(&empty_bar[s]);
+          }
+          if (ok) tc::umma_commit(&tfull_bar[acc]);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------ epilogue (4 warps)
+    const int q = warp & 3;  // tensor-memory lane quadrant this warp may read
+    const int n_valid = p.row0 + shape.rows;  // compact rows below this are real tokens
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; ok && u < shape.n_units; u += gridDim.x) {
+      const Unit w = decode_unit<MODE>(p, shape, u);
+      const int lrow = w.mb * BM + q * 32 + lane;  // row inside this launch's M range
+      // per-unit row state
+      float m_run = -INFINITY, s_run = 0.f, zt_val = 0.f;
+      bool zt_found = false;
+      int y = -1;
+      float gk = 0.f, lk = 0.f;
+      bool row_ok = false;
+      if (MODE == kFwd || MODE == kDz || MODE == kDh) {
+        const int k = p.row0 + lrow;
+        row_ok = k < n_valid;
+        if (row_ok) {
+          if (MODE == kFwd || MODE == kDh) y = p.targets[p.sel_idx[k]];
+          if (MODE == kDz || MODE == kDh) gk = p.g[k];
+          if (MODE == kDz) lk = p.lse[k];
+        }
+      } else {
+        row_ok = lrow < p.V;
+      }
+      for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt, ++tcount) {
+        const uint32_t acc = tcount & 1u;
+        const uint32_t aph = (tcount >> 1) & 1u;
+        // every lane waits (each needs the accumulator's writes visible), then the
+        // warp agrees on the outcome so the aligned tensor-memory loads stay converged
+        ok = __all_sync(0xFFFFFFFFu, tc::mbar_wait(&tfull_bar[acc], aph, abort_flag) ? 1 : 0) != 0;
+        if (!ok) break;
+        tc::fence_after_sync();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+        const int ncols = (MODE == kFwd || MODE == kDz) ? p.V : p.d;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          const int col0 = nt * BN + c * 32;
+          if (col0 >= ncols) break;  // warp-uniform
+          float v[32];
+          tc::tmem_ld32(taddr + c * 32, v);
+          if (MODE == kFwd) {
+            const int nv = ncols - col0 < 32 ? ncols - col0 : 32;
+            float cmax = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (j < nv) cmax = fmaxf(cmax, v[j]);
+            const float m_new = fmaxf(m_run, cmax);
+            const float mb2 = m_new * kLog2e;
+            float part = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (j < nv) part += fast_exp2(fmaf(v[j], kLog2e, -mb2));
+            s_run = s_run * fast_exp2((m_run - m_new) * kLog2e) + part;
+            m_run = m_new;
+            if (y >= col0 && y < col0 + 32) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j == y) zt_val = v[j];
+              zt_found = true;
+            }
+          } else if (MODE == kDz) {
+            const float nl2 = lk * kLog2e;
+            const float ng = -gk;
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float p0 = ng * fast_exp2(fmaf(v[2 * j], kLog2e, -nl2));
+              const float p1 = ng * fast_exp2(fmaf(v[2 * j + 1], kLog2e, -nl2));
+              packed[j] = pack_bf16(p0, p1);
+            }
+            __nv_bfloat16* dst = p.dZ + (size_t)lrow * p.ldz + col0;
+#pragma unroll
+            for (int g8 = 0; g8 < 4; ++g8)
+              if (col0 + 8 * g8 < ncols)
+                *reinterpret_cast<uint4*>(dst + 8 * g8) = make_uint4(
+                    packed[4 * g8], packed[4 * g8 + 1], packed[4 * g8 + 2], packed[4 * g8 + 3]);
+          } else if (MODE == kDh) {
+            if (row_ok) {
+              const int k = p.row0 + lrow;
+              const uint4* wsrc = reinterpret_cast<const uint4*>(p.W + (size_t)y * p.d + col0);
+              uint4* dst = reinterpret_cast<uint4*>(p.dH + (size_t)k * p.d + col0);
+#pragma unroll
+              for (int g8 = 0; g8 < 4; ++g8) {
+                const uint4 wv = __ldg(wsrc + g8);
+                const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+                uint32_t o[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const __nv_bfloat162 w2 = *reinterpret_cast<const __nv_bfloat162*>(&ww[e]);
+                  const float lo = fmaf(gk, __low2float(w2), v[8 * g8 + 2 * e]);
+                  const float hi = fmaf(gk, __high2float(w2), v[8 * g8 + 2 * e + 1]);
+                  o[e] = pack_bf16(lo, hi);
+                }
+                dst[g8] = make_uint4(o[0], o[1], o[2], o[3]);
+              }
+            }
+          } else {
+            if (row_ok) {
+              float4* dst = reinterpret_cast<float4*>(p.dW + (size_t)lrow * p.d + col0);
+#pragma unroll
+              for (int g4 = 0; g4 < 8; ++g4) {
+                float4 o = dst[g4];
+                o.x += v[4 * g4];
+                o.y += v[4 * g4 + 1];
+                o.z += v[4 * g4 + 2];
+                o.w += v[4 * g4 + 3];
+                dst[g4] = o;
+              }
+            }
+          }
+        }
+        tc::fence_before_sync();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&tempty_bar[acc]);
+      }
+      if (MODE == kFwd && ok && row_ok) {
+        const int k = p.row0 + lrow;
+        p.part_m[(size_t)w.sp * p.cap_pad + k] = m_run;
+        p.part_s[(size_t)w.sp * p.cap_pad + k] = s_run;
+        if (zt_found) p.zt[k] = zt_val;
+      }
+    }
+  }
+
+  tc::fence_before_sync();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag != 0u) atomicOr(p.status, NAT_DEV_TIMEOUT);
+  if (warp == 1) {
+    tc::fence_after_sync();
+    tc::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ----------------------------------------------------------- small kernels
+// Hc[k, :] = hidden[row(k), :] for k < n_sel, zero up to rows_pad, so that
+// every tile the tensor-core kernels touch holds finite values.
+__global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden,
+                                   const int32_t* __restrict__ sel_idx, int compact,
+                                   const int32_t* __restrict__ n_sel, int cap, int rows_pad, int d,
+                                   __nv_bfloat16* __restrict__ Hc) {
+  int n = *n_sel;
+  n = n < cap ? n : cap;
+  const int vec = d / 8;
+  for (int k = blockIdx.x; k < rows_pad; k += gridDim.x) {
+    uint4* dst = reinterpret_cast<uint4*>(Hc + (size_t)k * d);
+    if (k < n) {
+      const int64_t row = compact ? (int64_t)k : (int64_t)sel_idx[k];
+      const uint4* src = reinterpret_cast<const uint4*>(hidden + row * d);
+      for (int j = threadIdx.x; j < vec; j += blockDim.x) dst[j] = __ldg(src + j);
+    } else {
+      for (int j = threadIdx.x; j < vec; j += blockDim.x) dst[j] = make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+// Combine the per-split (max, sum-exp) pairs of each row, then the token's
+// log-probability and its share of the loss.
+__global__ void fwd_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_sel, int cap,
+                                    int n_splits, int cap_pad, const float* __restrict__ part_m,
+                                    const float* __restrict__ part_s, const float* __restrict__ zt,
+                                    float* __restrict__ logp, float* __restrict__ lse,
+                                    float* __restrict__ term) {
+  int n = *n_sel;
+  n = n < cap ? n : cap;
+  for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
+    float M = -INFINITY;
+    for (int sp = 0; sp < n_splits; ++sp) M = fmaxf(M, part_m[(size_t)sp * cap_pad + k]);
+    float S = 0.f;
+    for (int sp = 0; sp < n_splits; ++sp)
+      S += part_s[(size_t)sp * cap_pad + k] * expf(part_m[(size_t)sp * cap_pad + k] - M);
+    const float l = M + logf(S);
+    const float lp = zt[k] - l;
+    lse[k] = l;
+    logp[k] = lp;
+    float t, g;
+    token_eval(c, k, lp, 1.f, &t, &g);
+    term[k] = t;
+  }
+}
+
+// One-hot part of dW: dW[y_k, :] += g_k h_k.  Tokens that share a target meet
+// in the same row, hence atomics.
+__global__ void onehot_dw_kernel(const __nv_bfloat16* __restrict__ Hc,
+                                 const int32_t* __restrict__ targets,
+                                 const int32_t* __restrict__ sel_idx, const float* __restrict__ g,
+                                 const int32_t* __restrict__ n_sel, int cap, int d,
+                                 float* __restrict__ dW) {
+  int n = *n_sel;
+  n = n < cap ? n : cap;
+  for (int k = blockIdx.x; k < n; k += gridDim.x) {
+    const float gk = g[k];
+    if (gk == 0.f) continue;
+    const int y = targets[sel_idx[k]];
+    const __nv_bfloat16* h = Hc + (size_t)k * d;
+    float* dst = dW + (size_t)y * d;
+    for (int j = threadIdx.x; j < d; j += blockDim.x)
+      atomicAdd(dst + j, gk * __bfloat162float(h[j]));
+  }
+}
+
+// ------------------------------------------------------------- host side
+struct Layout {
+  int cap_pad, n_tiles, n_splits, chunk_rows, ldz;
+  size_t off_term, off_g, off_zt, off_pm, off_ps, off_hc, off_dz, total;
+};
+
+Layout make_layout(const nat_loss_params& p, int64_t cap) {
+  Layout L;
+  const int64_t c1 = cap > 0 ? cap : 1;
+  L.cap_pad = (int)((c1 + BM - 1) / BM * BM);
+  L.n_tiles = (p.V + BN - 1) / BN;
+  L.n_splits = (L.n_tiles + kTilesPerSplit - 1) / kTilesPerSplit;
+  L.chunk_rows = L.cap_pad < kChunkRows ? L.cap_pad : kChunkRows;
+  L.ldz = (p.V + 63) / 64 * 64;
+  size_t off = sizeof(WorkspaceHead);
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align_up(bytes, 1024);
+    return o;
+  };
+  L.off_term = take(sizeof(float) * L.cap_pad);
+  L.off_g = take(sizeof(float) * L.cap_pad);
+  L.off_zt = take(sizeof(float) * L.cap_pad);
+  L.off_pm = take(sizeof(float) * (size_t)L.cap_pad * L.n_splits);
+  L.off_ps = take(sizeof(float) * (size_t)L.cap_pad * L.n_splits);
+  off = align_up(off, 1024);
+  L.off_hc = take(sizeof(__nv_bfloat16) * (size_t)L.cap_pad * p.d);
+  L.off_dz = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * L.ldz);
+  L.total = off;
+  return L;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int get_encoder(EncodeTiledFn* out) {
+  static EncodeTiledFn cached = nullptr;
+  if (!cached) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    NAT_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (qres != cudaDriverEntryPointSuccess || !fn)
+      return fail(NAT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cached = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  *out = cached;
+  return NAT_OK;
+}
+
+// bf16 matrix [rows, inner] with the given row pitch; box = box_inner x box_rows
+// elements, 128-byte swizzle, out-of-range elements read as zero.
+int make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows,
+             uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_rows) {
+  EncodeTiledFn enc;
+  int s = get_encoder(&enc);
+  if (s != NAT_OK) return s;
+  const cuuint64_t dims[2] = {inner, rows};
+  const cuuint64_t strides[1] = {pitch_bytes};
+  const cuuint32_t box[2] = {box_inner, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(NAT_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return NAT_OK;
+}
+
+int sm_count(int* out) {
+  static int cached = 0;
+  if (!cached) {
+    int dev = 0;
+    NAT_CUDA(cudaGetDevice(&dev));
+    NAT_CUDA(cudaDeviceGetAttribute(&cached, cudaDevAttrMultiProcessorCount, dev));
+  }
+  *out = cached;
+  return NAT_OK;
+}
+
+template <int MODE>
+int launch_tc(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, int max_units,
+              cudaStream_t stream) {
+  static bool configured = false;
+  if (!configured) {
+    NAT_CUDA(cudaFuncSetAttribute(nat_tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)kSmemBytes));
+    configured = true;
+  }
+  int sms = 0;
+  int s = sm_count(&sms);
+  if (s != NAT_OK) return s;
+  const int grid = max_units < sms ? max_units : sms;
+  if (grid <= 0) return NAT_OK;
+  nat_tc_kernel<MODE><<<grid, kThreads, kSmemBytes, stream>>>(a, b, p);
+  NAT_LAUNCH_CHECK("nat_tc_kernel");
+  return NAT_OK;
+}
+
+TokenCtx make_ctx(const LossArgs& a) {
+  TokenCtx c;
+  c.targets = a.targets;
+  c.old_logp = a.old_logp;
+  c.adv = a.adv;
+  c.pi = a.pi;
+  c.cu_seqlens = a.cu_seqlens;
+  c.sel_idx = a.sel_idx;
+  c.sel_resp = a.sel_resp;
+  c.B = a.p.B;
+  c.clip_lo = a.p.clip_lo;
+  c.clip_hi = a.p.clip_hi;
+  return c;
+}
+
+struct Ws {
+  WorkspaceHead* head;
+  float *term, *g, *zt, *pm, *ps;
+  __nv_bfloat16 *hc, *dz;
+};
+
+Ws carve(void* ws, const Layout& L) {
+  char* b = reinterpret_cast<char*>(ws);
+  Ws w;
+  w.head = reinterpret_cast<WorkspaceHead*>(b);
+  w.term = reinterpret_cast<float*>(b + L.off_term);
+  w.g = reinterpret_cast<float*>(b + L.off_g);
+  w.zt = reinterpret_cast<float*>(b + L.off_zt);
+  w.pm = reinterpret_cast<float*>(b + L.off_pm);
+  w.ps = reinterpret_cast<float*>(b + L.off_ps);
+  w.hc = reinterpret_cast<__nv_bfloat16*>(b + L.off_hc);
+  w.dz = reinterpret_cast<__nv_bfloat16*>(b + L.off_dz);
+  return w;
+}
+
+TcParams base_params(const LossArgs& a, const Layout& L, const Ws& w) {
+  TcParams p{};
+  p.n_sel = a.n_sel;
+  p.cap = (int)a.cap;
+  p.row0 = 0;
+  p.chunk_rows = L.cap_pad;
+  p.d = a.p.d;
+  p.V = a.p.V;
+  p.n_splits = L.n_splits;
+  p.cap_pad = L.cap_pad;
+  p.targets = a.targets;
+  p.sel_idx = a.sel_idx;
+  p.part_m = w.pm;
+  p.part_s = w.ps;
+  p.zt = w.zt;
+  p.g = w.g;
+  p.lse = a.lse;
+  p.dZ = w.dz;
+  p.ldz = L.ldz;
+  p.W = reinterpret_cast<const __nv_bfloat16*>(a.W);
+  p.dH = reinterpret_cast<__nv_bfloat16*>(a.dHidden);
+  p.dW = a.dW;
+  p.status = &w.head->status;
+  return p;
+}
+
+int gather(const LossArgs& a, const Layout& L, const Ws& w) {
+  const int grid = L.cap_pad < 4096 ? L.cap_pad : 4096;
+  gather_rows_kernel<<<grid, 128, 0, a.stream>>>(
+      reinterpret_cast<const __nv_bfloat16*>(a.hidden), a.sel_idx, a.p.hidden_is_compact, a.n_sel,
+      (int)a.cap, L.cap_pad, a.p.d, w.hc);
+  NAT_LAUNCH_CHECK("gather_rows_kernel");
+  return NAT_OK;
+}
+
+}  // namespace
+
+size_t loss_bf16_workspace_bytes(const nat_loss_params& p, int64_t cap) {
+  return make_layout(p, cap).total;
+}
+
+int loss_bf16_fwd(const LossArgs& a) {
+  int s = require_sm100();
+  if (s != NAT_OK) return s;
+  const Layout L = make_layout(a.p, a.cap);
+  const Ws w = carve(a.workspace, L);
+  NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
+  const TokenCtx c = make_ctx(a);
+  if (a.cap > 0) {
+    if ((s = gather(a, L, w)) != NAT_OK) return s;
+    CUtensorMap mapA, mapB;
+    if ((s = make_map(&mapA, w.hc, a.p.d, L.cap_pad, (uint64_t)a.p.d * 2, BK, BM)) != NAT_OK) return s;
+    if ((s = make_map(&mapB, a.W, a.p.d, a.p.V, (uint64_t)a.p.d * 2, BK, BN)) != NAT_OK) return s;
+    const TcParams p = base_params(a, L, w);
+    if ((s = launch_tc<kFwd>(mapA, mapB, p, (L.cap_pad / BM) * L.n_splits, a.stream)) != NAT_OK)
+      return s;
+    const int grid = (int)((a.cap + 255) / 256 < 1184 ? (a.cap + 255) / 256 : 1184);
+    fwd_finalize_kernel<<<grid, 256, 0, a.stream>>>(c, a.n_sel, (int)a.cap, L.n_splits, L.cap_pad,
+                                                    w.pm, w.ps, w.zt, a.logp, a.lse, w.term);
+    NAT_LAUNCH_CHECK("fwd_finalize_kernel");
+  }
+  return launch_loss_reduce(w.term, a.n_sel, a.cap, a.loss, w.head, a.stream);
+}
+
+int loss_bf16_bwd(const LossArgs& a) {
+  int s = require_sm100();
+  if (s != NAT_OK) return s;
+  const Layout L = make_layout(a.p, a.cap);
+  const Ws w = carve(a.workspace, L);
+  NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
+  if (!a.p.accumulate_dW)
+    NAT_CUDA(cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)a.p.V * a.p.d, a.stream));
+  if (a.cap == 0) return NAT_OK;
+  const TokenCtx c = make_ctx(a);
+  if ((s = gather(a, L, w)) != NAT_OK) return s;
+  if ((s = launch_grad_coeff(c, a.logp, a.n_sel, a.cap, a.dloss, w.g, a.stream)) != NAT_OK) return s;
+
+  CUtensorMap mapHcK, mapWK, mapDzK, mapWmn, mapDzMn, mapHcMn;
+  const uint64_t dpitch = (uint64_t)a.p.d * 2, zpitch = (uint64_t)L.ldz * 2;
+  if ((s = make_map(&mapHcK, w.hc, a.p.d, L.cap_pad, dpitch, BK, BM)) != NAT_OK) return s;
+  if ((s = make_map(&mapWK, a.W, a.p.d, a.p.V, dpitch, BK, BN)) != NAT_OK) return s;
+  if ((s = make_map(&mapDzK, w.dz, a.p.V, L.chunk_rows, zpitch, BK, BM)) != NAT_OK) return s;
+  if ((s = make_map(&mapWmn, a.W, a.p.d, a.p.V, dpitch, 64, BK)) != NAT_OK) return s;
+  if ((s = make_map(&mapDzMn, w.dz, a.p.V, L.chunk_rows, zpitch, 64, BK)) != NAT_OK) return s;
+  if ((s = make_map(&mapHcMn, w.hc, a.p.d, L.cap_pad, dpitch, 64, BK)) != NAT_OK) return s;
+
+  const int nb_d = (a.p.d + BN - 1) / BN;
+  for (int row0 = 0; row0 < L.cap_pad; row0 += L.chunk_rows) {
+    TcParams p = base_params(a, L, w);
+    p.row0 = row0;
+    p.chunk_rows = L.chunk_rows;
+    const int mb = L.chunk_rows / BM;
+    if ((s = launch_tc<kDz>(mapHcK, mapWK, p, mb * L.n_splits, a.stream)) != NAT_OK) return s;
+    if ((s = launch_tc<kDh>(mapDzK, mapWmn, p, mb * nb_d, a.stream)) != NAT_OK) return s;
+    if ((s = launch_tc<kDw>(mapDzMn, mapHcMn, p, ((a.p.V + BM - 1) / BM) * nb_d, a.stream)) !=
+        NAT_OK)
+      return s;
+  }
+  const int grid = (int)(a.cap < 8192 ? a.cap : 8192);
+  onehot_dw_kernel<<<grid, 256, 0, a.stream>>>(w.hc, a.targets, a.sel_idx, w.g, a.n_sel,
+                                               (int)a.cap, a.p.d, a.dW);
+  NAT_LAUNCH_CHECK("onehot_dw_kernel");
+  return NAT_OK;
+}
+
+}  // namespace nat

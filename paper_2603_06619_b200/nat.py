@@ -1,0 +1,157 @@
+"""Python binding of the NAT C-ABI library (ctypes; argument marshalling only).
+
+Every function here has the name and the meaning of the C entry point it
+calls (see include/nat.h).  torch tensors supply device memory and the current
+CUDA stream; all arithmetic runs in the library's kernels.  There is no CPU
+fallback: loading fails loudly when the shared library is missing.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnat_b200.so")
+
+NAT_SEL_URS, NAT_SEL_RPC, NAT_SEL_DET = 0, 1, 2
+NAT_F32, NAT_BF16 = 0, 1
+NAT_DEV_TIMEOUT, NAT_DEV_CAPACITY = 1, 2
+
+SYMBOLS = (
+    "nat_status_string", "nat_last_error", "nat_version", "nat_grpo_adv", "nat_select",
+    "nat_compact_workspace_bytes", "nat_compact", "nat_policy_loss_workspace_bytes",
+    "nat_policy_loss_fwd", "nat_policy_loss_bwd",
+)
+
+
+class NatError(RuntimeError):
+    pass
+
+
+class SelectParams(ctypes.Structure):
+    _fields_ = [("mode", ctypes.c_int32), ("min_cut", ctypes.c_int32), ("p", ctypes.c_double),
+                ("beta", ctypes.c_double), ("seed", ctypes.c_uint64), ("offset", ctypes.c_uint64)]
+
+
+class LossParams(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("V", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("B", ctypes.c_int32), ("clip_lo", ctypes.c_float), ("clip_hi", ctypes.c_float),
+                ("hidden_is_compact", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def load():
+    """dlopen the library (built in-tree by ``build.build()``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise NatError(f"{LIB_PATH} is missing: run `python -m paper_2603_06619_b200.build` "
+                       "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    lib.nat_status_string.restype = ctypes.c_char_p
+    lib.nat_status_string.argtypes = [ctypes.c_int]
+    lib.nat_last_error.restype = ctypes.c_char_p
+    lib.nat_version.restype = ctypes.c_int
+    lib.nat_grpo_adv.argtypes = [i32, i32, vp, f32, vp, vp]
+    lib.nat_select.argtypes = [ctypes.POINTER(SelectParams), i32, vp, i64, vp, vp, vp, vp]
+    lib.nat_compact_workspace_bytes.restype = ctypes.c_size_t
+    lib.nat_compact_workspace_bytes.argtypes = [i64]
+    lib.nat_compact.argtypes = [i32, vp, i64, vp, vp, vp, vp, vp, i64, vp, ctypes.c_size_t, vp]
+    lib.nat_policy_loss_workspace_bytes.restype = ctypes.c_size_t
+    lib.nat_policy_loss_workspace_bytes.argtypes = [ctypes.POINTER(LossParams), i64]
+    lib.nat_policy_loss_fwd.argtypes = [ctypes.POINTER(LossParams)] + [vp] * 10 + [i64] + \
+        [vp] * 4 + [ctypes.c_size_t, vp]
+    lib.nat_policy_loss_bwd.argtypes = [ctypes.POINTER(LossParams)] + [vp] * 10 + [i64] + \
+        [vp] * 6 + [ctypes.c_size_t, vp]
+    for name in ("nat_grpo_adv", "nat_select", "nat_compact", "nat_policy_loss_fwd",
+                 "nat_policy_loss_bwd"):
+        getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(status):
+    if status != 0:
+        lib = load()
+        raise NatError(f"{lib.nat_status_string(status).decode()}: {lib.nat_last_error().decode()}")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous(), "tensors passed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def nat_grpo_adv(P, G, rewards, eps, adv):
+    _check(load().nat_grpo_adv(P, G, _ptr(rewards), eps, _ptr(adv), _stream()))
+
+
+def select_params(mode, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
+    mode = {"urs": NAT_SEL_URS, "rpc": NAT_SEL_RPC, "det": NAT_SEL_DET}.get(mode, mode)
+    return SelectParams(mode=mode, min_cut=min_cut, p=p, beta=beta, seed=seed, offset=offset)
+
+
+def nat_select(params, B, cu_seqlens, n_tot, mask, pi, cut_len):
+    _check(load().nat_select(ctypes.byref(params), B, _ptr(cu_seqlens), n_tot, _ptr(mask),
+                             _ptr(pi), _ptr(cut_len), _stream()))
+
+
+def nat_compact_workspace_bytes(n_tot):
+    return load().nat_compact_workspace_bytes(n_tot)
+
+
+def nat_compact(B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offsets, n_sel, cap, workspace):
+    _check(load().nat_compact(B, _ptr(cu_seqlens), n_tot, _ptr(mask), _ptr(sel_idx),
+                              _ptr(sel_resp), _ptr(sel_offsets), _ptr(n_sel), cap,
+                              _ptr(workspace), workspace.numel() * workspace.element_size(),
+                              _stream()))
+
+
+def loss_params(d, V, dtype, B, clip_lo=0.2, clip_hi=0.2, hidden_is_compact=False,
+                accumulate_dW=False):
+    dtype = {torch.float32: NAT_F32, torch.bfloat16: NAT_BF16}.get(dtype, dtype)
+    return LossParams(d=d, V=V, dtype=dtype, B=B, clip_lo=clip_lo, clip_hi=clip_hi,
+                      hidden_is_compact=int(hidden_is_compact), accumulate_dW=int(accumulate_dW))
+
+
+def nat_policy_loss_workspace_bytes(params, n_sel_cap):
+    return load().nat_policy_loss_workspace_bytes(ctypes.byref(params), n_sel_cap)
+
+
+def nat_policy_loss_fwd(params, hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx,
+                        sel_resp, n_sel, n_sel_cap, loss, logp, lse, workspace):
+    _check(load().nat_policy_loss_fwd(
+        ctypes.byref(params), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(old_logp), _ptr(adv),
+        _ptr(pi), _ptr(cu_seqlens), _ptr(sel_idx), _ptr(sel_resp), _ptr(n_sel), n_sel_cap,
+        _ptr(loss), _ptr(logp), _ptr(lse), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()))
+
+
+def nat_policy_loss_bwd(params, hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx,
+                        sel_resp, n_sel, n_sel_cap, logp, lse, dloss, dHidden, dW, workspace):
+    _check(load().nat_policy_loss_bwd(
+        ctypes.byref(params), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(old_logp), _ptr(adv),
+        _ptr(pi), _ptr(cu_seqlens), _ptr(sel_idx), _ptr(sel_resp), _ptr(n_sel), n_sel_cap,
+        _ptr(logp), _ptr(lse), _ptr(dloss), _ptr(dHidden), _ptr(dW), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()))
+
+
+def alloc_workspace(nbytes, device):
+    """256-byte aligned scratch (torch's caching allocator aligns to 512 bytes)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def device_status(workspace):
+    """The NAT_DEV_* bits the last loss call left in its workspace (synchronises)."""
+    return int(workspace[:4].view(torch.int32).item())

@@ -1,0 +1,122 @@
+"""GPU parity: policy-loss forward and backward against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_06619_b200 import nat
+from paper_2603_06619_b200 import workloads as wl
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["tiny", "tiny_rpc"])
+@pytest.mark.parametrize("seed", [0, 1])
+def test_tiny_fp32(name, seed):
+    out, _ = parity.run_case(wl.WORKLOADS[name], seed=seed)
+    assert out["dH_err"] < 1e-4 and out["dW_err"] < 1e-4
+
+
+def test_tiny_wide_noise_and_full_token():
+    # both clip branches fire with sigma = 0.3; p = 1 is full-token GRPO
+    w = wl.variant(wl.WORKLOADS["tiny"], old_noise=0.3)
+    out, ref = parity.run_case(w, seed=2)
+    assert (ref["g"] == 0).any() and (ref["g"] != 0).any()
+    parity.run_case(wl.variant(w, p=1.0), seed=2)
+    parity.run_case(wl.variant(w, sel_mode="det", beta=0.5), seed=2)
+
+
+@pytest.mark.parametrize("mode", ["urs", "rpc"])
+def test_mid_bf16(mode):
+    # 3 row tiles with a ragged tail, 20 vocabulary tiles with a ragged tail, 2 splits
+    w = wl.variant(wl.WORKLOADS["mid"], sel_mode=mode, min_cut=5)
+    parity.run_case(w, seed=0)
+
+
+def test_mid_bf16_peaked_softmax():
+    # logits with std ~8: exercises the running-max rescaling and makes the
+    # softmax part of the gradients as large as the one-hot part
+    w = wl.variant(wl.WORKLOADS["mid"], w_scale=0.5, old_noise=0.3)
+    out, ref = parity.run_case(w, seed=1)
+    assert out["dH_dense_err"] <= parity.TOL_DENSE
+
+
+def test_mid_bf16_multi_chunk_shapes():
+    # d not a multiple of 256 and V not a multiple of 8; more rows than one group of tiles
+    w = wl.variant(wl.WORKLOADS["mid"], d=320, V=3001, P=4, G=8, len_lo=60, len_hi=200, p=0.75)
+    parity.run_case(w, seed=3)
+
+
+def test_twin_0p6b():
+    parity.run_case(wl.WORKLOADS["twin_0p6b"], seed=0)
+
+
+def test_twin_8b():
+    parity.run_case(wl.WORKLOADS["twin_8b"], seed=0)
+
+
+def test_accumulate_dW_and_dloss():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = parity.gpu_step(w, batch, 0, 0)
+    base = st.dW.clone()
+    baseH = st.dH.clone()
+    dloss = torch.tensor([-2.0], device="cuda")
+    st.loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"],
+                batch["cu_seqlens"], dloss=dloss, accumulate_dW=True)
+    torch.cuda.synchronize()
+    n = int(st.n_sel.item())
+    assert parity.rel_fro(st.dW.cpu().numpy(), -base.cpu().numpy()) < 1e-2
+    assert parity.rel_fro(st.dH[:n].float().cpu().numpy(), -2 * baseH[:n].float().cpu().numpy()) < 1e-2
+
+
+def test_compact_hidden_layout():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=4, device="cuda")
+    nb = wl.to_numpy(batch)
+    ref_sel = parity.oracle_selection(w, nb, 4, 0)
+    idx = torch.from_numpy(ref_sel["sel_idx"]).long().cuda()
+    compact = dict(batch, hidden=batch["hidden"][idx].contiguous())
+    st = parity.gpu_step(w, compact, 4, 0, hidden_is_compact=True)
+    parity.check_selection(st, ref_sel, w)
+    parity.check_loss(st, ref_sel, nb, w)
+
+
+def test_empty_selection_and_reruns_are_deterministic():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = parity.gpu_step(w, batch, 0, 0)
+    loss1, logp1 = st.loss.clone(), st.logp.clone()
+    st.run(batch, w.sel_mode, p=w.p, seed=0)
+    torch.cuda.synchronize()
+    assert torch.equal(loss1, st.loss) and torch.equal(logp1, st.logp)
+    # nothing selected: loss 0 and zero dW
+    st.mask.zero_()
+    st.compact(batch["cu_seqlens"])
+    st.loss_fwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], batch["cu_seqlens"])
+    st.loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], batch["cu_seqlens"])
+    torch.cuda.synchronize()
+    assert int(st.n_sel.item()) == 0 and float(st.loss.item()) == 0.0
+    assert float(st.dW.abs().max().item()) == 0.0 and st.status() == 0
+
+
+def test_capacity_overflow_is_reported():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = parity.gpu_step(w, batch, 0, 0, backward=False, n_sel_cap=128)
+    assert int(st.n_sel.item()) > 128
+    assert st.status() & nat.NAT_DEV_CAPACITY
+
+
+def test_unsupported_shapes_are_rejected():
+    p = nat.loss_params(100, 512, torch.bfloat16, 8)      # d % 64 != 0
+    t = torch.zeros(1024, device="cuda")
+    ws = nat.alloc_workspace(1 << 20, "cuda")
+    with pytest.raises(nat.NatError):
+        nat.nat_policy_loss_fwd(p, t, t, t, t, t, t, t, t, t, t, 4, t, t, t, ws)
+    p = nat.loss_params(64, 512, torch.float32, 8)
+    tiny_ws = nat.alloc_workspace(256, "cuda")
+    with pytest.raises(nat.NatError):
+        nat.nat_policy_loss_fwd(p, t, t, t, t, t, t, t, t, t, t, 4096, t, t, t, tiny_ws)

@@ -1,0 +1,99 @@
+"""GPU parity: advantages, selection and compaction are bit-exact against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_06619_b200 import nat
+from paper_2603_06619_b200 import workloads as wl
+from paper_2603_06619_b200.step import NatStep
+
+from parity import MODE_ID
+
+pytestmark = pytest.mark.gpu
+
+
+def _select_compact(T, mode, P, G, seed=0, offset=0, p=0.5, min_cut=1, beta=0.5, cap=None,
+                    rewards=None):
+    T = np.asarray(T, dtype=np.int32)
+    cu = wl.cu_from_lengths(T)
+    n_tot = int(cu[-1])
+    st = NatStep(P, G, 64, 512, torch.float32, n_tot, n_sel_cap=cap, want_grads=False)
+    cu_d = torch.from_numpy(cu).cuda()
+    if rewards is None:
+        rewards = (np.random.default_rng(seed).random(P * G) < 0.4).astype(np.float32)
+    st.grpo_adv(torch.from_numpy(rewards).cuda())
+    st.select(cu_d, mode, p=p, min_cut=min_cut, beta=beta, seed=seed, offset=offset)
+    st.compact(cu_d)
+    torch.cuda.synchronize()
+    adv = oracle.grpo_adv(rewards, P, G, 1e-6)
+    mask, pi, cut = oracle.select(MODE_ID[mode], cu, p=p, min_cut=min_cut, beta=beta, seed=seed,
+                                  offset=offset)
+    si, sr, so, n = oracle.compact(mask, cu)
+    assert np.array_equal(st.adv.cpu().numpy().view(np.uint32), adv.view(np.uint32))
+    assert np.array_equal(st.mask[:n_tot].cpu().numpy(), mask)
+    assert np.array_equal(st.pi[:n_tot].cpu().numpy().view(np.uint32), pi.view(np.uint32))
+    if cut is not None:
+        assert np.array_equal(st.cut_len[:P * G].cpu().numpy(), cut)
+    assert int(st.n_sel.item()) == n
+    m = n if cap is None else min(n, cap)
+    assert np.array_equal(st.sel_idx[:m].cpu().numpy(), si[:m])
+    assert np.array_equal(st.sel_resp[:m].cpu().numpy(), sr[:m])
+    assert np.array_equal(st.sel_offsets.cpu().numpy(), so)
+    return n
+
+
+@pytest.mark.parametrize("mode", ["urs", "rpc", "det"])
+def test_tiny_lengths(mode):
+    w = wl.WORKLOADS["tiny"]
+    _select_compact(wl.make_lengths(w, 0), mode, w.P, w.G, seed=0)
+    _select_compact(wl.make_lengths(w, 1), mode, w.P, w.G, seed=1, offset=(7 << 32) + 3)
+
+
+@pytest.mark.parametrize("name", ["qwen3_0p6b", "qwen3_8b", "long_cot"])
+@pytest.mark.parametrize("mode", ["urs", "rpc", "det"])
+def test_config_lengths(name, mode):
+    w = wl.WORKLOADS[name]
+    n = _select_compact(wl.make_lengths(w, 0), mode, w.P, w.G, seed=0, p=0.5, min_cut=100)
+    assert n > 0
+
+
+@pytest.mark.parametrize("p", [0.25, 0.75, 1.0, 0.3, 1e-9])
+def test_urs_probabilities(p):
+    w = wl.WORKLOADS["qwen3_0p6b"]
+    _select_compact(wl.make_lengths(w, 3), "urs", w.P, w.G, seed=5, p=p)
+
+
+def test_edge_cases():
+    # empty responses at the start, middle and end; single tokens; chunk-edge sizes
+    _select_compact([0, 5, 0, 0, 3, 1, 0, 0], "urs", 2, 4, seed=2)
+    _select_compact([0, 5, 0, 0, 3, 1, 0, 0], "rpc", 2, 4, seed=2, min_cut=2)
+    _select_compact([0, 0, 0, 0], "rpc", 1, 4)
+    _select_compact([4096, 4096], "urs", 1, 2, seed=3)
+    _select_compact([4095, 1, 4096, 17], "det", 2, 2, seed=3)
+    _select_compact([1] * 64, "rpc", 8, 8, seed=4, min_cut=0)
+    _select_compact([30, 100, 101, 250], "rpc", 1, 4, seed=4, min_cut=100)
+    _select_compact([32768, 9], "rpc", 1, 2, seed=9, min_cut=1)
+
+
+def test_capacity_smaller_than_selection():
+    n = _select_compact([300, 200, 100, 50], "urs", 2, 2, seed=1, p=0.9, cap=64)
+    assert n > 64
+
+
+def test_rewards_real_valued():
+    r = np.random.default_rng(0).normal(size=48).astype(np.float32)
+    _select_compact([3] * 48, "urs", 6, 8, rewards=r)
+    _select_compact([3] * 48, "urs", 6, 8, rewards=np.full(48, 0.7, dtype=np.float32))
+
+
+def test_invalid_arguments_are_rejected():
+    cu = torch.zeros(3, dtype=torch.int32, device="cuda")
+    buf = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    pi = torch.zeros(16, dtype=torch.float32, device="cuda")
+    for kw in (dict(mode="urs", p=0.0), dict(mode="urs", p=1.5), dict(mode="det", beta=0.0),
+               dict(mode="rpc", min_cut=-1), dict(mode=7)):
+        with pytest.raises(nat.NatError):
+            nat.nat_select(nat.select_params(**kw), 2, cu, 0, buf, pi, cu)
+    with pytest.raises(nat.NatError):
+        nat.nat_grpo_adv(2, 0, pi, 1e-6, pi)
