@@ -1,0 +1,345 @@
+"""Benchmark of the partial-token GRPO policy-gradient step (NAT) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole path over one synthetic batch: advantages,
+selection, compaction, policy-loss forward and backward.  Rank 0 prints ONE
+JSON line.  `value` is selected tokens per second with inputs resident in HBM;
+`e2e` is the same with the step's inputs copied from pinned host memory and the
+loss read back inside the timed region.  `--impl reference` times the fp64 CPU
+oracle on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "selected tokens/sec, fused policy-loss fwd+bwd (Qwen3-8B head); % bf16 TC peak"
+UNIT = "selected tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count()
+
+
+# ---------------------------------------------------------------- CPU oracle
+def oracle_sample_rate(w, seed, rows, repeats=1):
+    """Selected tokens/s of the fp64 oracle (loss forward + backward) on `rows`
+    selected tokens of the workload's head (same d, V, dtype and value recipe)."""
+    import numpy as np
+    import oracle
+    from paper_2603_06619_b200 import workloads as wl
+
+    # a short batch with the workload's head: enough tokens that `rows` are selected
+    T = np.full(w.B, max(4, (2 * rows + w.B - 1) // w.B), dtype=np.int32)
+    batch = wl.to_numpy(wl.make_batch(w, seed=seed, lengths=T))
+    adv = oracle.grpo_adv(batch["rewards"], w.P, w.G, 1e-6)
+    mask, pi, _ = oracle.select(oracle.SEL_URS, batch["cu_seqlens"], p=1.0)
+    si, sr, _, _ = oracle.compact(mask, batch["cu_seqlens"])
+    si, sr = si[:rows], sr[:rows]
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.policy_loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"],
+                               adv, pi, batch["cu_seqlens"], si, sr)
+        times.append(time.perf_counter() - t0)
+    return len(si) / min(times), min(times), len(si), times
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows = args.ref_rows
+    for _ in range(args.warmup):
+        pass  # the oracle has no warm state worth building; keep the run short
+    rate, _, n, times = oracle_sample_rate(w, seed=0, rows=rows, repeats=max(1, args.steps))
+    ms = 1e3 * statistics.mean(times)
+    cores = host_cores()
+    sample = f"{n} selected rows of the {w.name} head per step (fp64 loss fwd+bwd, all of V)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": n / (ms / 1e3), "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "d": w.d, "V": w.V, "sample": sample},
+        "cpu_baseline": {"value": n / (ms / 1e3), "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": n / (ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------- ours
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2603_06619_b200 import build as _build
+    from paper_2603_06619_b200 import workloads as wl
+    from paper_2603_06619_b200.step import NatStep
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+
+    # Responses are independent, so ranks take disjoint batches (weak scaling):
+    # no collective sits on the data path.
+    seed = args.seed + rank
+    batch = wl.make_batch(w, seed=seed, device=dev)
+    n_tot = batch["n_tot"]
+    dtype = torch.float32 if w.dtype == "f32" else torch.bfloat16
+    st = NatStep(w.P, w.G, w.d, w.V, dtype, n_tot, device=dev)
+    cu = batch["cu_seqlens"]
+    sel = dict(mode=w.sel_mode, p=w.p, min_cut=w.min_cut, beta=w.beta, seed=seed)
+
+    def step(b, offset):
+        st.grpo_adv(b["rewards"])
+        st.select(cu, offset=offset, **sel)
+        st.compact(cu)
+        st.loss_fwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
+        st.loss_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(batch, i)
+    sync_all()
+    if st.status() != 0:
+        raise RuntimeError(f"device status {st.status()} after warm-up")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+
+    # ---- device-resident timing; forward and backward bracketed separately
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    n_sel_total = 0
+    sync_all()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        off = args.warmup + i
+        st.grpo_adv(batch["rewards"])
+        st.select(cu, offset=off, **sel)
+        st.compact(cu)
+        ev[i][0].record()
+        st.loss_fwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+        ev[i][1].record()
+        st.loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+        ev[i][2].record()
+    t_end.record()
+    sync_all()
+    elapsed_ms = t_begin.elapsed_time(t_end)
+    fwd_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    bwd_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    # selected tokens per step: selection with offsets warmup..warmup+K-1 (replayed, untimed)
+    for i in range(args.steps):
+        st.select(cu, offset=args.warmup + i, **sel)
+        st.compact(cu)
+        n_sel_total += int(st.n_sel.item())
+    status = st.status()
+    loss_val = float(st.loss.item())
+
+    # ---- end to end: the step's inputs come from pinned host memory
+    host = {k: batch[k].cpu().pin_memory() for k in ("hidden", "targets", "old_logp", "rewards")}
+    dev_in = {k: torch.empty_like(batch[k]) for k in host}
+    loss_host = torch.zeros(1, dtype=torch.float32).pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+
+    def e2e_step(offset):
+        for k in host:
+            dev_in[k].copy_(host[k], non_blocking=True)
+        b = dict(dev_in, W=batch["W"])
+        step(b, offset)
+        loss_host.copy_(st.loss, non_blocking=True)
+
+    e2e_step(0)
+    sync_all()
+    e_begin = torch.cuda.Event(enable_timing=True)
+    e_end = torch.cuda.Event(enable_timing=True)
+    e_begin.record()
+    for i in range(args.steps):
+        e2e_step(args.warmup + i)
+    e_end.record()
+    sync_all()
+    e2e_ms = e_begin.elapsed_time(e_end)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- max over ranks, totals over ranks
+    stats = torch.tensor([elapsed_ms, e2e_ms, fwd_ms, bwd_ms], dtype=torch.float64, device=dev)
+    total = torch.tensor([float(n_sel_total)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
+        dist.all_reduce(total, op=dist.ReduceOp.SUM)
+    elapsed_ms, e2e_ms, fwd_ms, bwd_ms = (float(x) for x in stats.tolist())
+    n_all = float(total.item())
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    n_step = n_sel_total / args.steps              # this rank's selected tokens per step
+    dV = float(w.d) * float(w.V)
+    # The step runs for seconds under the power cap, so the sustained tensor
+    # peak is the denominator; the burst figure is reported beside it.
+    peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    bwd_tflops = 4.0 * n_step * dV / (bwd_ms * 1e-3) / 1e12
+    fwd_tflops = 2.0 * n_step * dV / (fwd_ms * 1e-3) / 1e12
+    step_ms = elapsed_ms / args.steps
+    cap_pad = (n_tot + 127) // 128 * 128
+    n_chunks = (cap_pad + min(cap_pad, 8192) - 1) // min(cap_pad, 8192)
+    launches = 1 + (1 if w.sel_mode == "urs" else 2) + 3 + 4 + (3 + 3 * n_chunks)
+
+    line = {
+        "metric": METRIC, "value": n_all / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "P": w.P, "G": w.G, "d": w.d, "V": w.V,
+                   "selection": w.sel_mode, "p": w.p, "min_cut": w.min_cut,
+                   "n_tot_per_gpu": n_tot, "n_sel_per_step_per_gpu": n_step,
+                   "l2": "inputs larger than L2 (hidden and W_lm are GBs); no flush needed",
+                   "parallelism": f"dp{world} (independent batches, no collective)"},
+        "tflops_counted": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12,
+        "tflops_executed": 8.0 * n_step * dV / (step_ms * 1e-3) / 1e12,
+        "frac_of_peak_counted": {
+            "burst": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12 / float(peaks["bf16_tflops"]),
+            "sustained": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12 / peak,
+            "datasheet_2250": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12 / 2250.0},
+        "fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "loss": loss_val, "device_status": status,
+        "roofline": {
+            "kernel": "nat_tc_kernel<kDz|kDh|kDw> (the launches inside nat_policy_loss_bwd)",
+            "bound": "tensor", "achieved": bwd_tflops, "peak": peak, "unit": "TFLOP/s",
+            "frac": bwd_tflops / peak, "peak_source": f"{peak_kind} bf16_tflops_sustained",
+            "flops": "counted 4*N_sel*d*V per backward call (6*N_sel*d*V executed with the recompute)",
+            "traffic": None},
+        "roofline_fwd": {
+            "kernel": "nat_tc_kernel<kFwd>", "bound": "tensor", "achieved": fwd_tflops,
+            "peak": peak, "unit": "TFLOP/s", "frac": fwd_tflops / peak, "traffic": None},
+        "e2e": {"value": n_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": 4, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": launches * args.steps,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        rate, secs, n, _ = oracle_sample_rate(w, seed=0, rows=args.ref_rows)
+        line["cpu_baseline"] = {
+            "value": rate, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+            "sample": f"{n} selected rows of the {w.name} head (fp64 loss fwd+bwd over all of V) "
+                      f"in {secs:.1f} s"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3_8b")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--ref-rows", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2603_06619_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
