@@ -113,6 +113,35 @@ int nat_compact(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8
                 int64_t cap, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * nat_compact_static: nat_compact without a workspace argument.  (An addition
+ * of this library; the paper has no counterpart.)
+ *
+ * For callers that cannot obtain device memory at the point of the call: code
+ * running under a framework that has reserved the whole GPU for its own pool,
+ * plugin or callback contexts where cudaMalloc is forbidden or would
+ * synchronise the device, and tight inner loops that must not touch an
+ * allocator.  The scan scratch lives in a fixed array inside the library
+ * (64 KB of device memory per GPU that loads the library, held until the
+ * process exits), so the call allocates and frees nothing.
+ *
+ * Arguments, outputs and results are those of nat_compact.  Differences:
+ *   - n_tot may not exceed nat_compact_static_max_tokens() (67,108,864 tokens);
+ *     larger inputs return NAT_ERR_CAPACITY and enqueue nothing.
+ *   - The first call on each device looks up the array's device address (a
+ *     runtime query, not an allocation).  Make that first call outside any
+ *     stream capture.
+ *   - All calls on one GPU share the one array.  Calls whose kernels could run
+ *     at the same time (different streams without ordering) race on it and
+ *     give wrong results; order them on one stream or with events.  Nothing in
+ *     the array needs clearing between calls: each call overwrites what it
+ *     reads.
+ * ------------------------------------------------------------------------- */
+int64_t nat_compact_static_max_tokens(void);
+int nat_compact_static(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8_t* mask,
+                       int32_t* sel_idx, int32_t* sel_resp, int32_t* sel_offsets, int32_t* n_sel,
+                       int64_t cap, void* stream);
+
+/* ---------------------------------------------------------------------------
  * Policy loss over the selected tokens (ratio Eq. ratio, clipped surrogate
  * Eq. grpo-surrogate, sequence/group mean Eq. grpo-obj, Horvitz-Thompson
  * weights Eq. ht-estimator and Eq. rpc-ht; KL coefficient 0 as in the paper's

@@ -7,6 +7,8 @@
 // Floating-point steps that must agree bit for bit with a plain IEEE
 // evaluation use the explicit round-to-nearest intrinsics, which the compiler
 // never contracts into fused multiply-adds.
+#include <mutex>
+
 #include "nat_common.cuh"
 
 namespace nat {
@@ -430,6 +432,93 @@ int nat_compact(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8
   if (((uintptr_t)workspace & 255u) != 0)
     return fail(NAT_ERR_INVALID_ARG, "nat_compact: workspace must be 256-byte aligned");
   int32_t* chunk_count = reinterpret_cast<int32_t*>(workspace);
+  const int n_chunks = (int)((n_tot + kChunk - 1) / kChunk);
+  if (n_chunks > 0) {
+    compact_count_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(mask, n_tot, chunk_count);
+    NAT_LAUNCH_CHECK("compact_count_kernel");
+  }
+  compact_scan_kernel<<<1, 1024, 0, stream>>>(chunk_count, n_chunks, n_sel, sel_offsets, B);
+  NAT_LAUNCH_CHECK("compact_scan_kernel");
+  if (n_chunks > 0) {
+    compact_write_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(B, cu_seqlens, n_tot, mask,
+                                                               chunk_count, sel_idx, sel_resp,
+                                                               sel_offsets, cap);
+    NAT_LAUNCH_CHECK("compact_write_kernel");
+  } else if (B > 0) {
+    NAT_CUDA(cudaMemsetAsync(sel_offsets, 0, sizeof(int32_t) * (size_t)B, stream));
+  }
+  return NAT_OK;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------
+// nat_compact_static: the same compaction with its scan scratch held inside the
+// library instead of passed in.
+// ---------------------------------------------------------------------------
+namespace nat {
+namespace {
+
+// Chunk counts / offsets for up to kStaticMaxChunks chunks of 4096 tokens.
+// Lives in every CUDA context that loads this library, until the process ends.
+constexpr int kStaticMaxChunks = 16384;
+static __device__ __align__(256) int32_t g_compact_scratch[kStaticMaxChunks + 1];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+int32_t* g_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of g_compact_scratch on the current device.  In host code the
+// array's name is only a handle for the runtime, never a pointer a kernel could
+// use, so the address is asked for once per device and remembered.
+int static_scratch(int32_t** out) {
+  int dev = 0;
+  NAT_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices)
+    return fail(NAT_ERR_UNSUPPORTED, "nat_compact_static: device index %d not supported", dev);
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    NAT_CUDA(cudaGetSymbolAddress(&ptr, g_compact_scratch));
+    if (!ptr) return fail(NAT_ERR_CUDA, "nat_compact_static: scratch symbol has no address");
+    g_scratch_addr[dev] = static_cast<int32_t*>(ptr);
+  }
+  *out = g_scratch_addr[dev];
+  return NAT_OK;
+}
+
+}  // namespace
+}  // namespace nat
+
+extern "C" {
+
+int64_t nat_compact_static_max_tokens(void) {
+  return (int64_t)nat::kStaticMaxChunks * nat::kChunk;
+}
+
+int nat_compact_static(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8_t* mask,
+                       int32_t* sel_idx, int32_t* sel_resp, int32_t* sel_offsets, int32_t* n_sel,
+                       int64_t cap, void* stream_) {
+  using namespace nat;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (B < 0 || n_tot < 0 || cap < 0)
+    return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: negative size");
+  if (n_tot > nat_compact_static_max_tokens())
+    return fail(NAT_ERR_CAPACITY,
+                "nat_compact_static: n_tot = %lld exceeds the built-in scratch (at most %lld "
+                "tokens); use nat_compact with a caller-provided workspace",
+                (long long)n_tot, (long long)nat_compact_static_max_tokens());
+  if (!cu_seqlens || !sel_offsets || !n_sel)
+    return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: null pointer");
+  if (n_tot > 0 && !mask) return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: mask is null");
+  if (cap > 0 && (!sel_idx || !sel_resp))
+    return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: null list");
+  int32_t* chunk_count = nullptr;
+  int s = static_scratch(&chunk_count);
+  if (s != NAT_OK) return s;
+  // Every scratch entry this call reads is written earlier in the same call
+  // (counts by the first kernel, offsets and total by the scan), so nothing left
+  // by a previous call needs clearing.
   const int n_chunks = (int)((n_tot + kChunk - 1) / kChunk);
   if (n_chunks > 0) {
     compact_count_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(mask, n_tot, chunk_count);

@@ -20,7 +20,8 @@ NAT_DEV_TIMEOUT, NAT_DEV_CAPACITY = 1, 2
 SYMBOLS = (
     "nat_status_string", "nat_last_error", "nat_version", "nat_grpo_adv", "nat_select",
     "nat_compact_workspace_bytes", "nat_compact", "nat_policy_loss_workspace_bytes",
-    "nat_policy_loss_fwd", "nat_policy_loss_bwd",
+    "nat_policy_loss_fwd", "nat_policy_loss_bwd", "nat_compact_static",
+    "nat_compact_static_max_tokens",
 )
 
 
@@ -61,6 +62,9 @@ def load():
     lib.nat_compact_workspace_bytes.restype = ctypes.c_size_t
     lib.nat_compact_workspace_bytes.argtypes = [i64]
     lib.nat_compact.argtypes = [i32, vp, i64, vp, vp, vp, vp, vp, i64, vp, ctypes.c_size_t, vp]
+    lib.nat_compact_static_max_tokens.restype = ctypes.c_int64
+    lib.nat_compact_static.argtypes = [i32, vp, i64, vp, vp, vp, vp, vp, i64, vp]
+    lib.nat_compact_static.restype = ctypes.c_int
     lib.nat_policy_loss_workspace_bytes.restype = ctypes.c_size_t
     lib.nat_policy_loss_workspace_bytes.argtypes = [ctypes.POINTER(LossParams), i64]
     lib.nat_policy_loss_fwd.argtypes = [ctypes.POINTER(LossParams)] + [vp] * 10 + [i64] + \
@@ -116,6 +120,18 @@ def nat_compact(B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offsets, n_se
                               _ptr(sel_resp), _ptr(sel_offsets), _ptr(n_sel), cap,
                               _ptr(workspace), workspace.numel() * workspace.element_size(),
                               _stream()))
+
+
+def nat_compact_static_max_tokens():
+    return load().nat_compact_static_max_tokens()
+
+
+def nat_compact_static(B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offsets, n_sel, cap):
+    """nat_compact for callers that may not allocate: the scratch is a fixed array
+    inside the library (shared by all calls on the GPU, so do not overlap calls)."""
+    _check(load().nat_compact_static(B, _ptr(cu_seqlens), n_tot, _ptr(mask), _ptr(sel_idx),
+                                     _ptr(sel_resp), _ptr(sel_offsets), _ptr(n_sel), cap,
+                                     _stream()))
 
 
 def loss_params(d, V, dtype, B, clip_lo=0.2, clip_hi=0.2, hidden_is_compact=False,
