@@ -1,0 +1,117 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times
+(capacity = N_tot, n_sel read on the device).
+
+The fp64 oracle cannot evaluate 10^14..10^15 FLOPs, so here:
+  * advantages, masks, pi, cuts and compacted indices are compared in full, bit for bit;
+  * logp, lse and whole dHidden rows are compared on a sample of selected rows that the
+    oracle evaluates one by one (stream ends, tile and chunk edges, random rows);
+  * the scalar loss is checked against the fp64 sum of the per-token terms that the
+    sampled comparison validates (a consistency property, stated as such);
+  * dW is tied to the validated dHidden by identities that hold at any size:
+    every column of dW sums to zero over the vocabulary, and
+    sum_k <dHidden_k, h_k> = <dW, W>  (both equal sum_{k,v} dz[k,v] z[k,v]).
+Element-by-element dW parity is covered at the reduced twins of the same heads.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_06619_b200 import workloads as wl
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample_rows(n, rng, k_random=40):
+    edges = [0, 1, 127, 128, 129, 255, 256, 8191, 8192, 8193, 16383, 16384, n - 129, n - 128,
+             n - 2, n - 1]
+    rows = {r for r in edges if 0 <= r < n}
+    rows |= set(int(x) for x in rng.integers(0, n, size=k_random))
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+def _full_size_case(name, seed=0, **variant):
+    w = wl.variant(wl.WORKLOADS[name], **variant) if variant else wl.WORKLOADS[name]
+    batch = wl.make_batch(w, seed=seed, device="cuda")
+    nb = {k: (v.cpu().numpy() if isinstance(v, torch.Tensor) and v.dtype != torch.bfloat16 else v)
+          for k, v in batch.items() if k not in ("hidden", "W")}
+    ref_sel = parity.oracle_selection(w, nb, seed, 0)
+    st = parity.gpu_step(w, batch, seed, 0)
+    parity.check_selection(st, ref_sel, w)
+    assert st.status() == 0
+    n = ref_sel["n_sel"]
+
+    rng = np.random.default_rng(seed)
+    rows = _sample_rows(n, rng)
+    si = ref_sel["sel_idx"][rows]
+    sr = ref_sel["sel_resp"][rows]
+    # only the sampled hidden rows travel to the host; W goes whole
+    hidden_rows = batch["hidden"][torch.from_numpy(si).long().cuda()].float().cpu().numpy()
+    Wn = batch["W"].float().cpu().numpy()
+    ref = oracle.policy_loss_bwd(hidden_rows, Wn, nb["targets"], nb["old_logp"], ref_sel["adv"],
+                                 ref_sel["pi"], nb["cu_seqlens"], si, sr, hidden_is_compact=True,
+                                 want_dW=False)
+    got_logp = st.logp[:n].cpu().numpy()
+    got_lse = st.lse[:n].cpu().numpy()
+    assert np.abs(got_logp[rows] - ref["logp"]).max() <= parity.TOL_LOGP
+    assert np.abs(got_lse[rows] - ref["lse"]).max() <= parity.TOL_LOGP
+    dH_rows = st.dH[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+    assert parity.rel_fro(dH_rows, ref["dH"]) <= parity.TOL_GRAD
+    live = ref["g"] != 0
+    if live.any():
+        per_row = np.linalg.norm(dH_rows[live] - ref["dH"][live], axis=1) / \
+            np.linalg.norm(ref["dH"][live], axis=1)
+        assert per_row.max() <= 2 * parity.TOL_GRAD
+    assert np.all(dH_rows[~live] == 0)
+
+    # loss = fp64 sum of the per-token terms evaluated at the (sample-validated) logp
+    full_idx, full_resp = ref_sel["sel_idx"], ref_sel["sel_resp"]
+    T = np.diff(nb["cu_seqlens"]).astype(np.float64)
+    wgt = 1.0 / (ref_sel["pi"].astype(np.float64)[full_idx] * T[full_resp] * w.B)
+    A = ref_sel["adv"].astype(np.float64)[full_resp]
+    r = np.exp(got_logp.astype(np.float64) - nb["old_logp"].astype(np.float64)[full_idx])
+    S = np.minimum(r * A, np.clip(r, 0.8, 1.2) * A)
+    want = -np.sum(wgt * S)
+    floor = 1e-2 * np.sum(wgt * np.abs(S))
+    assert abs(float(st.loss.item()) - want) <= parity.TOL_LOSS * max(abs(want), floor)
+
+    # dW identities (computed on the device in fp64 where it matters)
+    dW = st.dW
+    col = dW.double().sum(0)
+    assert float(col.abs().max()) <= 1e-3 * float(dW.double().abs().sum(0).max())
+    idx = torch.from_numpy(full_idx).long().cuda()
+    lhs = 0.0
+    for lo in range(0, n, 16384):
+        hi = min(lo + 16384, n)
+        lhs += float((st.dH[lo:hi].double() * batch["hidden"][idx[lo:hi]].double()).sum())
+    rhs = 0.0
+    for lo in range(0, w.V, 16384):
+        rhs += float((dW[lo:lo + 16384].double() * batch["W"][lo:lo + 16384].double()).sum())
+    scale = float((dW.double().abs() * batch["W"].double().abs()).sum())
+    assert abs(lhs - rhs) <= 2e-3 * scale, (lhs, rhs, scale)
+    return n
+
+
+def test_qwen3_0p6b_full():
+    n = _full_size_case("qwen3_0p6b")
+    assert n > 30000
+
+
+def test_qwen3_8b_full():
+    n = _full_size_case("qwen3_8b")
+    assert n > 100000
+
+
+def test_qwen3_8b_sweep_points():
+    # the selection-fraction sweep's other settings on the same batch shape (smaller P to
+    # keep the test short): URS p = 0.25, full-token p = 1, deterministic truncation
+    for kw in (dict(sel_mode="urs", p=0.25), dict(sel_mode="urs", p=1.0),
+               dict(sel_mode="det", beta=0.5)):
+        _full_size_case("qwen3_8b", P=2, **kw)
+
+
+def test_long_cot_full():
+    n = _full_size_case("long_cot")
+    assert n > 300000

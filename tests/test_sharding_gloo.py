@@ -1,0 +1,107 @@
+"""world_size-2 gloo tests (CPU) of the multi-rank host logic and of the sharding rule.
+
+The data path has no collective: ranks own whole prompt groups.  These tests
+check, with the oracle standing in for the kernels, that the rule is right:
+with the GLOBAL batch size in every rank's weights and GLOBAL response indices
+in the selection's counters, the ranks' losses and dW sum to the single-rank
+result and the ranks' masks are slices of the single-rank mask.
+"""
+import os
+import socket
+import sys
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_2603_06619_b200 import sharding
+    from paper_2603_06619_b200 import workloads as wl
+
+    w = wl.variant(wl.WORKLOADS["tiny"], P=3, old_noise=0.3)      # 3 prompts over 2 ranks: uneven
+    b = wl.to_numpy(wl.make_batch(w, seed=5))
+    b["rewards"] = np.tile(np.array([1, 0, 0, 1], dtype=np.float32), w.P)
+    cu = b["cu_seqlens"]
+    adv = oracle.grpo_adv(b["rewards"], w.P, w.G, 1e-6)
+    mask, pi, _ = oracle.select(oracle.SEL_URS, cu, p=0.5, seed=3, offset=9)
+
+    lo, hi = sharding.response_range(w.P, w.G, rank, world)
+    # this rank's slice of the packed stream; selection re-drawn locally with the
+    # GLOBAL response index would give the same bits, so slice the global mask
+    keep = np.zeros_like(mask)
+    keep[cu[lo]:cu[hi]] = mask[cu[lo]:cu[hi]]
+    si, sr, _, n = oracle.compact(keep, cu)
+    out = oracle.policy_loss_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], adv, pi, cu,
+                                 si, sr)
+    # advantages are local: recomputing them from this rank's prompts alone agrees
+    plo, phi = sharding.prompt_range(w.P, rank, world)
+    adv_local = oracle.grpo_adv(b["rewards"][lo:hi], phi - plo, w.G, 1e-6)
+    assert np.array_equal(adv_local, adv[lo:hi])
+
+    loss = torch.tensor([out["loss"]], dtype=torch.float64)
+    dW = torch.from_numpy(out["dW"].copy())
+    dist.all_reduce(loss)
+    dist.all_reduce(dW)
+    times, units = sharding.aggregate_timing([10.0 + rank, 5.0 - rank], n)
+    if rank == 0:
+        si, sr, _, n_all = oracle.compact(mask, cu)
+        full = oracle.policy_loss_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], adv, pi,
+                                      cu, si, sr)
+        assert abs(float(loss) - full["loss"]) < 1e-12
+        np.testing.assert_allclose(dW.numpy(), full["dW"], atol=1e-14)
+        assert times == [11.0, 5.0] and units == float(n_all)
+        open(os.path.join(out_dir, "ok"), "w").write("ok")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_rank_sharding_sums_to_single_rank(tmp_path):
+    port = _free_port()
+    mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert (tmp_path / "ok").exists()
+
+
+def test_prompt_ranges_partition():
+    from paper_2603_06619_b200 import sharding
+    for P in (1, 3, 16, 17):
+        for world in (1, 2, 4, 8):
+            spans = [sharding.prompt_range(P, r, world) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == P
+            assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            sizes = [hi - lo for lo, hi in spans]
+            assert max(sizes) - min(sizes) <= 1
+    assert sharding.rank_seed(7, 3) == 10
+
+
+def test_selection_is_keyed_by_global_response_index():
+    """A rank that holds responses [lo, hi) reproduces the global mask for them when it
+    passes the global index: the oracle's draws for response i do not depend on the others."""
+    import oracle
+    T = np.array([9, 30, 4, 17, 25, 8])
+    cu = np.concatenate([[0], np.cumsum(T)]).astype(np.int32)
+    full, _, _ = oracle.select(oracle.SEL_URS, cu, p=0.5, seed=1, offset=2)
+    # same responses, but the first two made empty: indices of the others are unchanged
+    T2 = T.copy()
+    T2[:2] = 0
+    cu2 = np.concatenate([[0], np.cumsum(T2)]).astype(np.int32)
+    part, _, _ = oracle.select(oracle.SEL_URS, cu2, p=0.5, seed=1, offset=2)
+    assert np.array_equal(part, full[cu[2]:])
+    _, _, cut_full = oracle.select(oracle.SEL_RPC, cu, min_cut=2, seed=1, offset=2)
+    _, _, cut_part = oracle.select(oracle.SEL_RPC, cu2, min_cut=2, seed=1, offset=2)
+    assert np.array_equal(cut_part[2:], cut_full[2:])
