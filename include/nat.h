@@ -46,6 +46,8 @@ typedef enum {
 /* Bits of the device status word (first 4 bytes of a loss workspace). */
 #define NAT_DEV_TIMEOUT 1u  /* a bounded mbarrier wait gave up; outputs are invalid */
 #define NAT_DEV_CAPACITY 2u /* *n_sel exceeded n_sel_cap; surplus rows were ignored */
+#define NAT_DEV_FALLBACK 4u /* informational: nat_policy_loss_fwd_bwd redid some row chunk with
+                               the two-pass kernels (results are valid) */
 
 const char* nat_status_string(int status);
 const char* nat_last_error(void); /* host string, valid until the thread's next failing call */
@@ -210,6 +212,28 @@ int nat_policy_loss_bwd(const nat_loss_params* params /* host */, const void* hi
                         int64_t n_sel_cap, const float* logp, const float* lse,
                         const float* dloss, void* dHidden, float* dW, void* workspace,
                         size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Forward and backward in one call (same definitions and outputs as
+ * nat_policy_loss_fwd followed by nat_policy_loss_bwd: Eq. ratio,
+ * Eq. grpo-surrogate, Eq. grpo-obj, Eq. ht-estimator / Eq. rpc-ht and their
+ * gradient, Appendix A).  The bf16 path evaluates the projection S = H W^T once
+ * per block of rows instead of twice: it keeps the softmax numerators
+ * exp(S - mref) of at most 8192 rows in the workspace (mref = the row's largest
+ * logit over the first 256 vocabulary entries), and the per-row factors
+ * (1/sum, g) are applied outside the two gradient contractions.  If some logit
+ * exceeds its row's mref by more than 60 the block is redone by the two-pass
+ * kernels and NAT_DEV_FALLBACK is set; results are the same either way within
+ * the rounding of bf16 staging.  Arguments as in the two separate calls;
+ * outputs loss, logp, lse, dHidden, dW.
+ * ------------------------------------------------------------------------- */
+int nat_policy_loss_fwd_bwd(const nat_loss_params* params /* host */, const void* hidden,
+                            const void* W, const int32_t* targets, const float* old_logp,
+                            const float* adv, const float* pi, const int32_t* cu_seqlens,
+                            const int32_t* sel_idx, const int32_t* sel_resp,
+                            const int32_t* n_sel, int64_t n_sel_cap, const float* dloss,
+                            float* loss, float* logp, float* lse, void* dHidden, float* dW,
+                            void* workspace, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

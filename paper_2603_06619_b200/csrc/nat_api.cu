@@ -30,7 +30,8 @@ int require_sm100() {
   return NAT_OK;
 }
 
-static int validate(const char* who, const nat_loss_params* p, const LossArgs& a, bool bwd) {
+static int validate(const char* who, const nat_loss_params* p, const LossArgs& a, bool bwd,
+                    bool fwd = true) {
   if (!p) return fail(NAT_ERR_INVALID_ARG, "%s: params is null", who);
   if (p->d <= 0 || p->V <= 0 || p->B <= 0)
     return fail(NAT_ERR_INVALID_ARG, "%s: d, V and B must be positive", who);
@@ -43,7 +44,7 @@ static int validate(const char* who, const nat_loss_params* p, const LossArgs& a
   if (!a.hidden || !a.W || !a.targets || !a.old_logp || !a.adv || !a.pi || !a.cu_seqlens ||
       !a.sel_idx || !a.sel_resp || !a.n_sel || !a.logp || !a.lse)
     return fail(NAT_ERR_INVALID_ARG, "%s: null pointer", who);
-  if (!bwd && !a.loss) return fail(NAT_ERR_INVALID_ARG, "%s: loss is null", who);
+  if ((!bwd || fwd) && !a.loss) return fail(NAT_ERR_INVALID_ARG, "%s: loss is null", who);
   if (bwd && (!a.dHidden || !a.dW)) return fail(NAT_ERR_INVALID_ARG, "%s: null gradient", who);
   if (p->dtype == NAT_BF16) {
     if (p->d % 64 != 0)
@@ -117,9 +118,28 @@ int nat_policy_loss_bwd(const nat_loss_params* params, const void* hidden, const
   a.cap = n_sel_cap; a.logp = const_cast<float*>(logp); a.lse = const_cast<float*>(lse);
   a.dloss = dloss; a.dHidden = dHidden; a.dW = dW;
   a.workspace = workspace; a.workspace_bytes = workspace_bytes; a.stream = (cudaStream_t)stream;
-  int s = nat::validate("nat_policy_loss_bwd", params, a, true);
+  int s = nat::validate("nat_policy_loss_bwd", params, a, true, false);
   if (s != NAT_OK) return s;
   return params->dtype == NAT_F32 ? nat::loss_f32_bwd(a) : nat::loss_bf16_bwd(a);
+}
+
+int nat_policy_loss_fwd_bwd(const nat_loss_params* params, const void* hidden, const void* W,
+                            const int32_t* targets, const float* old_logp, const float* adv,
+                            const float* pi, const int32_t* cu_seqlens, const int32_t* sel_idx,
+                            const int32_t* sel_resp, const int32_t* n_sel, int64_t n_sel_cap,
+                            const float* dloss, float* loss, float* logp, float* lse,
+                            void* dHidden, float* dW, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+  nat::LossArgs a{};
+  if (params) a.p = *params;
+  a.hidden = hidden; a.W = W; a.targets = targets; a.old_logp = old_logp; a.adv = adv; a.pi = pi;
+  a.cu_seqlens = cu_seqlens; a.sel_idx = sel_idx; a.sel_resp = sel_resp; a.n_sel = n_sel;
+  a.cap = n_sel_cap; a.loss = loss; a.logp = logp; a.lse = lse; a.dloss = dloss;
+  a.dHidden = dHidden; a.dW = dW;
+  a.workspace = workspace; a.workspace_bytes = workspace_bytes; a.stream = (cudaStream_t)stream;
+  int s = nat::validate("nat_policy_loss_fwd_bwd", params, a, true, true);
+  if (s != NAT_OK) return s;
+  return params->dtype == NAT_F32 ? nat::loss_f32_fwd_bwd(a) : nat::loss_bf16_fwd_bwd(a);
 }
 
 }  // extern "C"

@@ -64,9 +64,11 @@ struct LossArgs {
 size_t loss_f32_workspace_bytes(const nat_loss_params& p, int64_t cap);
 int loss_f32_fwd(const LossArgs& a);
 int loss_f32_bwd(const LossArgs& a);
+int loss_f32_fwd_bwd(const LossArgs& a);
 
 size_t loss_bf16_workspace_bytes(const nat_loss_params& p, int64_t cap);
 int loss_bf16_fwd(const LossArgs& a);
 int loss_bf16_bwd(const LossArgs& a);
+int loss_bf16_fwd_bwd(const LossArgs& a);
 
 }  // namespace nat

@@ -10,6 +10,18 @@
 //                                        the bounded scratch dZ[chunk, V].
 //   kDh   dH = dZ W   (rows x d, K = V)  epilogue: + g W[y] (one-hot term) -> bf16.
 //   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 read-modify-write.
+//   kE    S = Hc W^T  single-pass variant  epilogue: E = exp(S - mref) -> bf16 into the
+//                                        same scratch, row sums of E, target pick.
+//
+// Two ways through the backward.  The two-pass route recomputes S (kDz) from the
+// forward's lse.  The single-pass route (nat_policy_loss_fwd_bwd) computes S once per
+// row chunk: kE stores the softmax numerators relative to a per-row reference mref (the
+// row maximum over the first vocabulary tile, from a one-tile kFwd launch), the row
+// scalars lse, g and c = -g / sum(E) follow, and because they are per-row they move out
+// of the contractions: dH = c (E W) + g W[y] (scaled in kDh's epilogue) and
+// dW += E^T (c h) (rows of Hc scaled into Hs).  A chunk in which some logit exceeds its
+// row's reference by more than 60 (E would leave the fp32/bf16 range) is redone by the
+// two-pass kernels, which are launched predicated on the chunk's flag.
 //
 // Roles per CTA (192 threads): warp 0 issues TMA loads into a 4-stage shared
 // memory ring, warp 1 issues tcgen05.mma into one of two 128x256 fp32
@@ -37,7 +49,9 @@ constexpr int kTilesPerSplit = 16;                 // vocabulary tiles per work 
 constexpr int kChunkRows = 8192;                   // rows of the dZ scratch
 constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 
-enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3 };
+enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3, kE = 4 };
+
+constexpr float kWindow = 60.f;  // largest S - mref the single-pass route accepts
 
 struct TcParams {
   const int32_t* n_sel;
@@ -60,6 +74,12 @@ struct TcParams {
   __nv_bfloat16* dH;
   float* dW;
   uint32_t* status;
+  const float* mref;       // kE: per-row reference
+  const float* row_scale;  // kDh: per-row factor on the accumulator (null = 1)
+  int b_row0;              // kDw: first row of the B operand's tensor map for this launch
+  const int32_t* flag;     // predicate: the launch does nothing unless
+  int run_if;              //   (*flag != 0) == run_if   (flag == null: always runs)
+  int32_t* ovf;            // kE: set to 1 when the window is exceeded
 };
 
 struct Unit {
@@ -84,8 +104,9 @@ __device__ __forceinline__ Shape make_shape(const TcParams& p) {
   n = n < p.cap ? n : p.cap;
   int rows = n - p.row0;
   rows = rows < 0 ? 0 : (rows > p.chunk_rows ? p.chunk_rows : rows);
+  if (p.flag != nullptr && ((*p.flag != 0) ? 1 : 0) != p.run_if) rows = 0;
   s.rows = rows;
-  if (MODE == kFwd || MODE == kDz) {
+  if (MODE == kFwd || MODE == kDz || MODE == kE) {
     s.mblocks = (rows + BM - 1) / BM;
     s.nblocks = (p.V + BN - 1) / BN;
     s.n_units = s.mblocks * p.n_splits;
@@ -110,7 +131,7 @@ __device__ __forceinline__ Shape make_shape(const TcParams& p) {
 template <int MODE>
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Shape& s, int u) {
   Unit w;
-  if (MODE == kFwd || MODE == kDz) {
+  if (MODE == kFwd || MODE == kDz || MODE == kE) {
     const int per_group = kGroupRows * p.n_splits;
     const int grp = u / per_group;
     const int rem = u - grp * per_group;
@@ -204,7 +225,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             uint8_t* a_dst = smem + (size_t)s * kStageBytes;
             uint8_t* b_dst = a_dst + kABytes;
             tc::mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
-            if (MODE == kFwd || MODE == kDz) {
+            if (MODE == kFwd || MODE == kDz || MODE == kE) {
               tc::tma_load_2d(a_dst, &mapA, &full_bar[s], kb * BK, p.row0 + w.mb * BM);
               tc::tma_load_2d(b_dst, &mapB, &full_bar[s], kb * BK, nt * BN);
             } else if (MODE == kDh) {
@@ -221,7 +242,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 #pragma unroll
               for (int j = 0; j < BN / 64; ++j)
                 tc::tma_load_2d(b_dst + j * kBoxBytes, &mapB, &full_bar[s], nt * BN + j * 64,
-                                p.row0 + kb * BK);
+                                p.b_row0 + kb * BK);
             }
           }
         }
@@ -295,15 +316,17 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       float m_run = -INFINITY, s_run = 0.f, zt_val = 0.f;
       bool zt_found = false;
       int y = -1;
-      float gk = 0.f, lk = 0.f;
-      bool row_ok = false;
-      if (MODE == kFwd || MODE == kDz || MODE == kDh) {
+      float gk = 0.f, lk = 0.f, scale = 1.f;
+      bool row_ok = false, over = false;
+      if (MODE != kDw) {
         const int k = p.row0 + lrow;
         row_ok = k < n_valid;
         if (row_ok) {
-          if (MODE == kFwd || MODE == kDh) y = p.targets[p.sel_idx[k]];
+          if (MODE == kFwd || MODE == kDh || MODE == kE) y = p.targets[p.sel_idx[k]];
           if (MODE == kDz || MODE == kDh) gk = p.g[k];
           if (MODE == kDz) lk = p.lse[k];
+          if (MODE == kE) lk = p.mref[k];
+          if (MODE == kDh && p.row_scale != nullptr) scale = p.row_scale[k];
         }
       } else {
         row_ok = lrow < p.V;
@@ -317,7 +340,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         if (!ok) break;
         tc::fence_after_sync();
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
-        const int ncols = (MODE == kFwd || MODE == kDz) ? p.V : p.d;
+        const int ncols = (MODE == kFwd || MODE == kDz || MODE == kE) ? p.V : p.d;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           const int col0 = nt * BN + c * 32;
@@ -344,6 +367,35 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 if (col0 + j == y) zt_val = v[j];
               zt_found = true;
             }
+          } else if (MODE == kE) {
+            const int nv = ncols - col0 < 32 ? ncols - col0 : 32;
+            const float nm2 = lk * kLog2e;
+            const float live = row_ok ? 1.f : 0.f;
+            float part = 0.f, tmax = -INFINITY;
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float t0 = fmaf(v[2 * j], kLog2e, -nm2);
+              const float t1 = fmaf(v[2 * j + 1], kLog2e, -nm2);
+              float e0 = live * fast_exp2(t0), e1 = live * fast_exp2(t1);
+              if (2 * j < nv) { part += e0; tmax = fmaxf(tmax, t0); }
+              if (2 * j + 1 < nv) { part += e1; tmax = fmaxf(tmax, t1); }
+              packed[j] = pack_bf16(e0, e1);
+            }
+            s_run += part;
+            if (row_ok && tmax > kWindow * kLog2e) over = true;
+            if (y >= col0 && y < col0 + 32) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j == y) zt_val = v[j];
+              zt_found = true;
+            }
+            __nv_bfloat16* dst = p.dZ + (size_t)lrow * p.ldz + col0;
+#pragma unroll
+            for (int g8 = 0; g8 < 4; ++g8)
+              if (col0 + 8 * g8 < ncols)
+                *reinterpret_cast<uint4*>(dst + 8 * g8) = make_uint4(
+                    packed[4 * g8], packed[4 * g8 + 1], packed[4 * g8 + 2], packed[4 * g8 + 3]);
           } else if (MODE == kDz) {
             const float nl2 = lk * kLog2e;
             const float ng = -gk;
@@ -373,8 +425,8 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                   const __nv_bfloat162 w2 = *reinterpret_cast<const __nv_bfloat162*>(&ww[e]);
-                  const float lo = fmaf(gk, __low2float(w2), v[8 * g8 + 2 * e]);
-                  const float hi = fmaf(gk, __high2float(w2), v[8 * g8 + 2 * e + 1]);
+                  const float lo = fmaf(gk, __low2float(w2), scale * v[8 * g8 + 2 * e]);
+                  const float hi = fmaf(gk, __high2float(w2), scale * v[8 * g8 + 2 * e + 1]);
                   o[e] = pack_bf16(lo, hi);
                 }
                 dst[g8] = make_uint4(o[0], o[1], o[2], o[3]);
@@ -405,6 +457,12 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         p.part_s[(size_t)w.sp * p.cap_pad + k] = s_run;
         if (zt_found) p.zt[k] = zt_val;
       }
+      if (MODE == kE && ok && row_ok) {
+        const int k = p.row0 + lrow;
+        p.part_s[(size_t)w.sp * p.cap_pad + k] = s_run;
+        if (zt_found) p.zt[k] = zt_val;
+        if (over) *p.ovf = 1;
+      }
     }
   }
 
@@ -418,6 +476,10 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 }
 
 // ----------------------------------------------------------- small kernels
+__device__ __forceinline__ bool predicate_off(const int32_t* flag, int run_if) {
+  return flag != nullptr && ((*flag != 0) ? 1 : 0) != run_if;
+}
+
 // Hc[k, :] = hidden[row(k), :] for k < n_sel, zero up to rows_pad, so that
 // every tile the tensor-core kernels touch holds finite values.
 __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden,
@@ -439,16 +501,24 @@ __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden,
   }
 }
 
-// Combine the per-split (max, sum-exp) pairs of each row, then the token's
-// log-probability and its share of the loss.
+// Rows [row0, row0 + rows_max): combine the per-split (max, sum-exp) pairs of each row,
+// then the token's log-probability, its share of the loss and (when g_out is given) its
+// gradient coefficient.
 __global__ void fwd_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_sel, int cap,
-                                    int n_splits, int cap_pad, const float* __restrict__ part_m,
+                                    int row0, int rows_max, int n_splits, int cap_pad,
+                                    const float* __restrict__ part_m,
                                     const float* __restrict__ part_s, const float* __restrict__ zt,
                                     float* __restrict__ logp, float* __restrict__ lse,
-                                    float* __restrict__ term) {
+                                    float* __restrict__ term, float* __restrict__ g_out,
+                                    const float* __restrict__ dloss,
+                                    const int32_t* __restrict__ flag, int run_if) {
+  if (predicate_off(flag, run_if)) return;
   int n = *n_sel;
   n = n < cap ? n : cap;
-  for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
+  const int end = n < row0 + rows_max ? n : row0 + rows_max;
+  const float dl = dloss ? *dloss : 1.f;
+  for (int k = row0 + blockIdx.x * blockDim.x + threadIdx.x; k < end;
+       k += gridDim.x * blockDim.x) {
     float M = -INFINITY;
     for (int sp = 0; sp < n_splits; ++sp) M = fmaxf(M, part_m[(size_t)sp * cap_pad + k]);
     float S = 0.f;
@@ -459,9 +529,81 @@ __global__ void fwd_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_se
     lse[k] = l;
     logp[k] = lp;
     float t, g;
-    token_eval(c, k, lp, 1.f, &t, &g);
+    token_eval(c, k, lp, dl, &t, &g);
     term[k] = t;
+    if (g_out) g_out[k] = g;
   }
+}
+
+// Single-pass route, rows [row0, row0 + chunk_rows) (one block per row): from the row
+// sums of E = exp(z - mref): lse = mref + log sum, logp, loss term, g, the row factor
+// c = -g / sum, and Hs[row - row0, :] = c * Hc[row, :].  Rows past the last selected
+// token are zero-filled in Hs.
+__global__ void fused_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_sel, int cap,
+                                      int row0, int chunk_rows, int n_splits, int cap_pad,
+                                      const float* __restrict__ mref,
+                                      const float* __restrict__ part_s,
+                                      const float* __restrict__ zt, const float* __restrict__ dloss,
+                                      float* __restrict__ logp, float* __restrict__ lse,
+                                      float* __restrict__ term, float* __restrict__ g_out,
+                                      float* __restrict__ cs, const __nv_bfloat16* __restrict__ Hc,
+                                      __nv_bfloat16* __restrict__ Hs, int d,
+                                      const int32_t* __restrict__ flag) {
+  if (predicate_off(flag, 0)) return;
+  __shared__ float c_s;
+  int n = *n_sel;
+  n = n < cap ? n : cap;
+  const float dl = dloss ? *dloss : 1.f;
+  const int vec = d / 8;
+  for (int r = blockIdx.x; r < chunk_rows; r += gridDim.x) {
+    const int k = row0 + r;
+    if (k >= n && r >= ((n - row0 + BM - 1) / BM) * BM) break;  // beyond the tiles in use
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float cv = 0.f;
+      if (k < n) {
+        float S = 0.f;
+        for (int sp = 0; sp < n_splits; ++sp) S += part_s[(size_t)sp * cap_pad + k];
+        const float l = mref[k] + logf(S);
+        const float lp = zt[k] - l;
+        lse[k] = l;
+        logp[k] = lp;
+        float t, g;
+        token_eval(c, k, lp, dl, &t, &g);
+        term[k] = t;
+        g_out[k] = g;
+        cv = -g / S;
+        cs[k] = cv;
+      }
+      c_s = cv;
+    }
+    __syncthreads();
+    const float cv = c_s;
+    uint4* dst = reinterpret_cast<uint4*>(Hs + (size_t)r * d);
+    if (cv == 0.f) {
+      for (int j = threadIdx.x; j < vec; j += blockDim.x) dst[j] = make_uint4(0, 0, 0, 0);
+    } else {
+      const uint4* src = reinterpret_cast<const uint4*>(Hc + (size_t)k * d);
+      for (int j = threadIdx.x; j < vec; j += blockDim.x) {
+        const uint4 hv = src[j];
+        const uint32_t in[4] = {hv.x, hv.y, hv.z, hv.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&in[e]);
+          o[e] = pack_bf16(cv * __low2float(h2), cv * __high2float(h2));
+        }
+        dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
+  }
+}
+
+// Records that some chunk left the single-pass window (informational status bit).
+__global__ void note_fallback_kernel(const int32_t* __restrict__ ovf, int n_chunks,
+                                     uint32_t* status) {
+  for (int c = threadIdx.x; c < n_chunks; c += blockDim.x)
+    if (ovf[c] != 0) atomicOr(status, NAT_DEV_FALLBACK);
 }
 
 // One-hot part of dW: dW[y_k, :] += g_k h_k.  Tokens that share a target meet
@@ -486,8 +628,9 @@ __global__ void onehot_dw_kernel(const __nv_bfloat16* __restrict__ Hc,
 
 // ------------------------------------------------------------- host side
 struct Layout {
-  int cap_pad, n_tiles, n_splits, chunk_rows, ldz;
-  size_t off_term, off_g, off_zt, off_pm, off_ps, off_hc, off_dz, total;
+  int cap_pad, n_tiles, n_splits, chunk_rows, n_chunks, ldz;
+  size_t off_term, off_g, off_zt, off_pm, off_ps, off_mref, off_cs, off_ovf, off_hc, off_hs,
+      off_dz, total;
 };
 
 Layout make_layout(const nat_loss_params& p, int64_t cap) {
@@ -497,6 +640,7 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   L.n_tiles = (p.V + BN - 1) / BN;
   L.n_splits = (L.n_tiles + kTilesPerSplit - 1) / kTilesPerSplit;
   L.chunk_rows = L.cap_pad < kChunkRows ? L.cap_pad : kChunkRows;
+  L.n_chunks = (L.cap_pad + L.chunk_rows - 1) / L.chunk_rows;
   L.ldz = (p.V + 63) / 64 * 64;
   size_t off = sizeof(WorkspaceHead);
   auto take = [&](size_t bytes) {
@@ -509,8 +653,12 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   L.off_zt = take(sizeof(float) * L.cap_pad);
   L.off_pm = take(sizeof(float) * (size_t)L.cap_pad * L.n_splits);
   L.off_ps = take(sizeof(float) * (size_t)L.cap_pad * L.n_splits);
+  L.off_mref = take(sizeof(float) * L.cap_pad);
+  L.off_cs = take(sizeof(float) * L.cap_pad);
+  L.off_ovf = take(sizeof(int32_t) * L.n_chunks);
   off = align_up(off, 1024);
   L.off_hc = take(sizeof(__nv_bfloat16) * (size_t)L.cap_pad * p.d);
+  L.off_hs = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * p.d);
   L.off_dz = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * L.ldz);
   L.total = off;
   return L;
@@ -602,8 +750,9 @@ TokenCtx make_ctx(const LossArgs& a) {
 
 struct Ws {
   WorkspaceHead* head;
-  float *term, *g, *zt, *pm, *ps;
-  __nv_bfloat16 *hc, *dz;
+  float *term, *g, *zt, *pm, *ps, *mref, *cs;
+  int32_t* ovf;
+  __nv_bfloat16 *hc, *hs, *dz;
 };
 
 Ws carve(void* ws, const Layout& L) {
@@ -615,7 +764,11 @@ Ws carve(void* ws, const Layout& L) {
   w.zt = reinterpret_cast<float*>(b + L.off_zt);
   w.pm = reinterpret_cast<float*>(b + L.off_pm);
   w.ps = reinterpret_cast<float*>(b + L.off_ps);
+  w.mref = reinterpret_cast<float*>(b + L.off_mref);
+  w.cs = reinterpret_cast<float*>(b + L.off_cs);
+  w.ovf = reinterpret_cast<int32_t*>(b + L.off_ovf);
   w.hc = reinterpret_cast<__nv_bfloat16*>(b + L.off_hc);
+  w.hs = reinterpret_cast<__nv_bfloat16*>(b + L.off_hs);
   w.dz = reinterpret_cast<__nv_bfloat16*>(b + L.off_dz);
   return w;
 }
@@ -643,6 +796,12 @@ TcParams base_params(const LossArgs& a, const Layout& L, const Ws& w) {
   p.dH = reinterpret_cast<__nv_bfloat16*>(a.dHidden);
   p.dW = a.dW;
   p.status = &w.head->status;
+  p.mref = w.mref;
+  p.row_scale = nullptr;
+  p.b_row0 = 0;
+  p.flag = nullptr;
+  p.run_if = 0;
+  p.ovf = nullptr;
   return p;
 }
 
@@ -652,6 +811,54 @@ int gather(const LossArgs& a, const Layout& L, const Ws& w) {
       reinterpret_cast<const __nv_bfloat16*>(a.hidden), a.sel_idx, a.p.hidden_is_compact, a.n_sel,
       (int)a.cap, L.cap_pad, a.p.d, w.hc);
   NAT_LAUNCH_CHECK("gather_rows_kernel");
+  return NAT_OK;
+}
+
+struct Maps {
+  CUtensorMap hcK, wK, dzK, wMn, dzMn, hcMn, hsMn;
+};
+
+int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
+  int s;
+  const uint64_t dpitch = (uint64_t)a.p.d * 2, zpitch = (uint64_t)L.ldz * 2;
+  if ((s = make_map(&m->hcK, w.hc, a.p.d, L.cap_pad, dpitch, BK, BM)) != NAT_OK) return s;
+  if ((s = make_map(&m->wK, a.W, a.p.d, a.p.V, dpitch, BK, BN)) != NAT_OK) return s;
+  if ((s = make_map(&m->dzK, w.dz, a.p.V, L.chunk_rows, zpitch, BK, BM)) != NAT_OK) return s;
+  if ((s = make_map(&m->wMn, a.W, a.p.d, a.p.V, dpitch, 64, BK)) != NAT_OK) return s;
+  if ((s = make_map(&m->dzMn, w.dz, a.p.V, L.chunk_rows, zpitch, 64, BK)) != NAT_OK) return s;
+  if ((s = make_map(&m->hcMn, w.hc, a.p.d, L.cap_pad, dpitch, 64, BK)) != NAT_OK) return s;
+  if ((s = make_map(&m->hsMn, w.hs, a.p.d, L.chunk_rows, dpitch, 64, BK)) != NAT_OK) return s;
+  return NAT_OK;
+}
+
+int finalize_grid(int rows) {
+  const int g = (rows + 255) / 256;
+  return g < 1 ? 1 : (g > 1184 ? 1184 : g);
+}
+
+// The three two-pass backward launches for rows [row0, row0 + chunk_rows); `flag`
+// (may be null) predicates them on the chunk having left the single-pass window.
+int launch_two_pass_chunk(const LossArgs& a, const Layout& L, const Ws& w, const Maps& m,
+                          int row0, const int32_t* flag) {
+  int s;
+  TcParams p = base_params(a, L, w);
+  p.row0 = row0;
+  p.chunk_rows = L.chunk_rows;
+  p.b_row0 = row0;
+  p.flag = flag;
+  p.run_if = 1;
+  const int mb = L.chunk_rows / BM;
+  const int nb_d = (a.p.d + BN - 1) / BN;
+  if ((s = launch_tc<kDz>(m.hcK, m.wK, p, mb * L.n_splits, a.stream)) != NAT_OK) return s;
+  if ((s = launch_tc<kDh>(m.dzK, m.wMn, p, mb * nb_d, a.stream)) != NAT_OK) return s;
+  return launch_tc<kDw>(m.dzMn, m.hcMn, p, ((a.p.V + BM - 1) / BM) * nb_d, a.stream);
+}
+
+int launch_onehot(const LossArgs& a, const Ws& w) {
+  const int grid = (int)(a.cap < 8192 ? a.cap : 8192);
+  onehot_dw_kernel<<<grid, 256, 0, a.stream>>>(w.hc, a.targets, a.sel_idx, w.g, a.n_sel,
+                                               (int)a.cap, a.p.d, a.dW);
+  NAT_LAUNCH_CHECK("onehot_dw_kernel");
   return NAT_OK;
 }
 
@@ -676,9 +883,9 @@ int loss_bf16_fwd(const LossArgs& a) {
     const TcParams p = base_params(a, L, w);
     if ((s = launch_tc<kFwd>(mapA, mapB, p, (L.cap_pad / BM) * L.n_splits, a.stream)) != NAT_OK)
       return s;
-    const int grid = (int)((a.cap + 255) / 256 < 1184 ? (a.cap + 255) / 256 : 1184);
-    fwd_finalize_kernel<<<grid, 256, 0, a.stream>>>(c, a.n_sel, (int)a.cap, L.n_splits, L.cap_pad,
-                                                    w.pm, w.ps, w.zt, a.logp, a.lse, w.term);
+    fwd_finalize_kernel<<<finalize_grid((int)a.cap), 256, 0, a.stream>>>(
+        c, a.n_sel, (int)a.cap, 0, L.cap_pad, L.n_splits, L.cap_pad, w.pm, w.ps, w.zt, a.logp,
+        a.lse, w.term, nullptr, nullptr, nullptr, 0);
     NAT_LAUNCH_CHECK("fwd_finalize_kernel");
   }
   return launch_loss_reduce(w.term, a.n_sel, a.cap, a.loss, w.head, a.stream);
@@ -696,33 +903,78 @@ int loss_bf16_bwd(const LossArgs& a) {
   const TokenCtx c = make_ctx(a);
   if ((s = gather(a, L, w)) != NAT_OK) return s;
   if ((s = launch_grad_coeff(c, a.logp, a.n_sel, a.cap, a.dloss, w.g, a.stream)) != NAT_OK) return s;
+  Maps m;
+  if ((s = make_maps(a, L, w, &m)) != NAT_OK) return s;
+  for (int row0 = 0; row0 < L.cap_pad; row0 += L.chunk_rows)
+    if ((s = launch_two_pass_chunk(a, L, w, m, row0, nullptr)) != NAT_OK) return s;
+  return launch_onehot(a, w);
+}
 
-  CUtensorMap mapHcK, mapWK, mapDzK, mapWmn, mapDzMn, mapHcMn;
-  const uint64_t dpitch = (uint64_t)a.p.d * 2, zpitch = (uint64_t)L.ldz * 2;
-  if ((s = make_map(&mapHcK, w.hc, a.p.d, L.cap_pad, dpitch, BK, BM)) != NAT_OK) return s;
-  if ((s = make_map(&mapWK, a.W, a.p.d, a.p.V, dpitch, BK, BN)) != NAT_OK) return s;
-  if ((s = make_map(&mapDzK, w.dz, a.p.V, L.chunk_rows, zpitch, BK, BM)) != NAT_OK) return s;
-  if ((s = make_map(&mapWmn, a.W, a.p.d, a.p.V, dpitch, 64, BK)) != NAT_OK) return s;
-  if ((s = make_map(&mapDzMn, w.dz, a.p.V, L.chunk_rows, zpitch, 64, BK)) != NAT_OK) return s;
-  if ((s = make_map(&mapHcMn, w.hc, a.p.d, L.cap_pad, dpitch, 64, BK)) != NAT_OK) return s;
-
-  const int nb_d = (a.p.d + BN - 1) / BN;
-  for (int row0 = 0; row0 < L.cap_pad; row0 += L.chunk_rows) {
-    TcParams p = base_params(a, L, w);
-    p.row0 = row0;
-    p.chunk_rows = L.chunk_rows;
+// Forward and backward in one call with a single pass over S per row chunk.
+int loss_bf16_fwd_bwd(const LossArgs& a) {
+  int s = require_sm100();
+  if (s != NAT_OK) return s;
+  const Layout L = make_layout(a.p, a.cap);
+  const Ws w = carve(a.workspace, L);
+  NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
+  NAT_CUDA(cudaMemsetAsync(w.ovf, 0, sizeof(int32_t) * L.n_chunks, a.stream));
+  if (!a.p.accumulate_dW)
+    NAT_CUDA(cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)a.p.V * a.p.d, a.stream));
+  const TokenCtx c = make_ctx(a);
+  if (a.cap > 0) {
+    if ((s = gather(a, L, w)) != NAT_OK) return s;
+    Maps m;
+    if ((s = make_maps(a, L, w, &m)) != NAT_OK) return s;
     const int mb = L.chunk_rows / BM;
-    if ((s = launch_tc<kDz>(mapHcK, mapWK, p, mb * L.n_splits, a.stream)) != NAT_OK) return s;
-    if ((s = launch_tc<kDh>(mapDzK, mapWmn, p, mb * nb_d, a.stream)) != NAT_OK) return s;
-    if ((s = launch_tc<kDw>(mapDzMn, mapHcMn, p, ((a.p.V + BM - 1) / BM) * nb_d, a.stream)) !=
-        NAT_OK)
-      return s;
+    const int nb_d = (a.p.d + BN - 1) / BN;
+    // Row references: the row maximum over the first vocabulary tile (a kFwd launch that
+    // sees a vocabulary of one tile and writes its running maximum to mref).
+    {
+      TcParams p = base_params(a, L, w);
+      p.V = a.p.V < BN ? a.p.V : BN;
+      p.n_splits = 1;
+      p.part_m = w.mref;
+      if ((s = launch_tc<kFwd>(m.hcK, m.wK, p, L.cap_pad / BM, a.stream)) != NAT_OK) return s;
+    }
+    for (int ci = 0; ci < L.n_chunks; ++ci) {
+      const int row0 = ci * L.chunk_rows;
+      int32_t* ovf = w.ovf + ci;
+      TcParams p = base_params(a, L, w);
+      p.row0 = row0;
+      p.chunk_rows = L.chunk_rows;
+      p.ovf = ovf;
+      if ((s = launch_tc<kE>(m.hcK, m.wK, p, mb * L.n_splits, a.stream)) != NAT_OK) return s;
+      fused_finalize_kernel<<<L.chunk_rows < 2048 ? L.chunk_rows : 2048, 128, 0, a.stream>>>(
+          c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_splits, L.cap_pad, w.mref, w.ps, w.zt,
+          a.dloss, a.logp, a.lse, w.term, w.g, w.cs, w.hc, w.hs, a.p.d, ovf);
+      NAT_LAUNCH_CHECK("fused_finalize_kernel");
+      p.ovf = nullptr;
+      p.flag = ovf;
+      p.run_if = 0;
+      p.row_scale = w.cs;
+      p.b_row0 = 0;  // Hs is local to the chunk
+      if ((s = launch_tc<kDh>(m.dzK, m.wMn, p, mb * nb_d, a.stream)) != NAT_OK) return s;
+      if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, p, ((a.p.V + BM - 1) / BM) * nb_d, a.stream)) !=
+          NAT_OK)
+        return s;
+      // Predicated redo of the chunk by the two-pass kernels (no-ops unless *ovf != 0).
+      TcParams pf = base_params(a, L, w);
+      pf.row0 = row0;
+      pf.chunk_rows = L.chunk_rows;
+      pf.flag = ovf;
+      pf.run_if = 1;
+      if ((s = launch_tc<kFwd>(m.hcK, m.wK, pf, mb * L.n_splits, a.stream)) != NAT_OK) return s;
+      fwd_finalize_kernel<<<finalize_grid(L.chunk_rows), 256, 0, a.stream>>>(
+          c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_splits, L.cap_pad, w.pm, w.ps, w.zt,
+          a.logp, a.lse, w.term, w.g, a.dloss, ovf, 1);
+      NAT_LAUNCH_CHECK("fwd_finalize_kernel");
+      if ((s = launch_two_pass_chunk(a, L, w, m, row0, ovf)) != NAT_OK) return s;
+    }
+    note_fallback_kernel<<<1, 128, 0, a.stream>>>(w.ovf, L.n_chunks, &w.head->status);
+    NAT_LAUNCH_CHECK("note_fallback_kernel");
+    if ((s = launch_onehot(a, w)) != NAT_OK) return s;
   }
-  const int grid = (int)(a.cap < 8192 ? a.cap : 8192);
-  onehot_dw_kernel<<<grid, 256, 0, a.stream>>>(w.hc, a.targets, a.sel_idx, w.g, a.n_sel,
-                                               (int)a.cap, a.p.d, a.dW);
-  NAT_LAUNCH_CHECK("onehot_dw_kernel");
-  return NAT_OK;
+  return launch_loss_reduce(w.term, a.n_sel, a.cap, a.loss, w.head, a.stream);
 }
 
 }  // namespace nat

@@ -254,4 +254,11 @@ int loss_f32_bwd(const LossArgs& a) {
   return NAT_OK;
 }
 
+// The fp32 path has no single-pass variant: forward, then backward.
+int loss_f32_fwd_bwd(const LossArgs& a) {
+  int s = loss_f32_fwd(a);
+  if (s != NAT_OK) return s;
+  return loss_f32_bwd(a);
+}
+
 }  // namespace nat

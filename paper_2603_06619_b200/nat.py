@@ -15,13 +15,13 @@ LIB_PATH = os.path.join(_HERE, "libnat_b200.so")
 
 NAT_SEL_URS, NAT_SEL_RPC, NAT_SEL_DET = 0, 1, 2
 NAT_F32, NAT_BF16 = 0, 1
-NAT_DEV_TIMEOUT, NAT_DEV_CAPACITY = 1, 2
+NAT_DEV_TIMEOUT, NAT_DEV_CAPACITY, NAT_DEV_FALLBACK = 1, 2, 4
 
 SYMBOLS = (
     "nat_status_string", "nat_last_error", "nat_version", "nat_grpo_adv", "nat_select",
     "nat_compact_workspace_bytes", "nat_compact", "nat_policy_loss_workspace_bytes",
     "nat_policy_loss_fwd", "nat_policy_loss_bwd", "nat_compact_static",
-    "nat_compact_static_max_tokens",
+    "nat_compact_static_max_tokens", "nat_policy_loss_fwd_bwd",
 )
 
 
@@ -71,8 +71,10 @@ def load():
         [vp] * 4 + [ctypes.c_size_t, vp]
     lib.nat_policy_loss_bwd.argtypes = [ctypes.POINTER(LossParams)] + [vp] * 10 + [i64] + \
         [vp] * 6 + [ctypes.c_size_t, vp]
+    lib.nat_policy_loss_fwd_bwd.argtypes = [ctypes.POINTER(LossParams)] + [vp] * 10 + [i64] + \
+        [vp] * 7 + [ctypes.c_size_t, vp]
     for name in ("nat_grpo_adv", "nat_select", "nat_compact", "nat_policy_loss_fwd",
-                 "nat_policy_loss_bwd"):
+                 "nat_policy_loss_bwd", "nat_policy_loss_fwd_bwd"):
         getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -160,6 +162,16 @@ def nat_policy_loss_bwd(params, hidden, W, targets, old_logp, adv, pi, cu_seqlen
         ctypes.byref(params), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(old_logp), _ptr(adv),
         _ptr(pi), _ptr(cu_seqlens), _ptr(sel_idx), _ptr(sel_resp), _ptr(n_sel), n_sel_cap,
         _ptr(logp), _ptr(lse), _ptr(dloss), _ptr(dHidden), _ptr(dW), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _stream()))
+
+
+def nat_policy_loss_fwd_bwd(params, hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx,
+                            sel_resp, n_sel, n_sel_cap, dloss, loss, logp, lse, dHidden, dW,
+                            workspace):
+    _check(load().nat_policy_loss_fwd_bwd(
+        ctypes.byref(params), _ptr(hidden), _ptr(W), _ptr(targets), _ptr(old_logp), _ptr(adv),
+        _ptr(pi), _ptr(cu_seqlens), _ptr(sel_idx), _ptr(sel_resp), _ptr(n_sel), n_sel_cap,
+        _ptr(dloss), _ptr(loss), _ptr(logp), _ptr(lse), _ptr(dHidden), _ptr(dW), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream()))
 
 

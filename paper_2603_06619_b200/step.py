@@ -65,12 +65,24 @@ class NatStep:
                                 cu_seqlens, self.sel_idx, self.sel_resp, self.n_sel, self.cap,
                                 self.logp, self.lse, dloss, self.dH, self.dW, self.loss_ws)
 
-    def run(self, batch, mode, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0, backward=True):
+    def loss_fwd_bwd(self, hidden, W, targets, old_logp, cu_seqlens, dloss=None,
+                     accumulate_dW=False):
+        self.params.accumulate_dW = int(accumulate_dW)
+        nat.nat_policy_loss_fwd_bwd(self.params, hidden, W, targets, old_logp, self.adv, self.pi,
+                                    cu_seqlens, self.sel_idx, self.sel_resp, self.n_sel, self.cap,
+                                    dloss, self.loss, self.logp, self.lse, self.dH, self.dW,
+                                    self.loss_ws)
+
+    def run(self, batch, mode, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0, backward=True,
+            fused=False):
         """All steps of the path on one batch (a dict from ``workloads.make_batch``)."""
         cu = batch["cu_seqlens"]
         self.grpo_adv(batch["rewards"])
         self.select(cu, mode, p=p, min_cut=min_cut, beta=beta, seed=seed, offset=offset)
         self.compact(cu)
+        if fused:
+            self.loss_fwd_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+            return
         self.loss_fwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
         if backward:
             self.loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)

@@ -42,11 +42,11 @@ def oracle_selection(w, nb, seed, offset, eps=1e-6):
                 n_sel=n)
 
 
-def gpu_step(w, batch, seed, offset, backward=True, n_sel_cap=None, **kw):
+def gpu_step(w, batch, seed, offset, backward=True, n_sel_cap=None, fused=False, **kw):
     dtype = torch.float32 if w.dtype == "f32" else torch.bfloat16
     st = NatStep(w.P, w.G, w.d, w.V, dtype, batch["n_tot"], n_sel_cap=n_sel_cap, **kw)
     st.run(batch, w.sel_mode, p=w.p, min_cut=w.min_cut, beta=w.beta, seed=seed, offset=offset,
-           backward=backward)
+           backward=backward, fused=fused)
     torch.cuda.synchronize()
     return st
 
@@ -74,7 +74,7 @@ def check_loss(st, ref_sel, nb, w, backward=True, hidden_is_compact=False, clip=
     ref = fn(hidden, nb["W"], nb["targets"], nb["old_logp"], ref_sel["adv"], ref_sel["pi"],
              nb["cu_seqlens"], ref_sel["sel_idx"], ref_sel["sel_resp"], clip_lo=clip[0],
              clip_hi=clip[1], hidden_is_compact=hidden_is_compact)
-    assert st.status() == 0
+    assert st.status() & ~4 == 0      # the informational fallback bit may be set
     got_logp = st.logp[:n].cpu().numpy()
     got_lse = st.lse[:n].cpu().numpy()
     assert np.abs(got_logp - ref["logp"]).max(initial=0) <= TOL_LOGP
@@ -107,10 +107,10 @@ def check_loss(st, ref_sel, nb, w, backward=True, hidden_is_compact=False, clip=
     return out, ref
 
 
-def run_case(w, seed=0, offset=0, backward=True, device="cuda", **batch_kw):
+def run_case(w, seed=0, offset=0, backward=True, device="cuda", fused=False, **batch_kw):
     batch = wl.make_batch(w, seed=seed, device=device, **batch_kw)
     nb = wl.to_numpy(batch)
     ref_sel = oracle_selection(w, nb, seed, offset)
-    st = gpu_step(w, batch, seed, offset, backward=backward)
+    st = gpu_step(w, batch, seed, offset, backward=backward, fused=fused)
     check_selection(st, ref_sel, w)
     return check_loss(st, ref_sel, nb, w, backward=backward)

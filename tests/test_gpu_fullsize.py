@@ -32,13 +32,13 @@ def _sample_rows(n, rng, k_random=40):
     return np.array(sorted(rows), dtype=np.int64)
 
 
-def _full_size_case(name, seed=0, **variant):
+def _full_size_case(name, seed=0, fused=False, **variant):
     w = wl.variant(wl.WORKLOADS[name], **variant) if variant else wl.WORKLOADS[name]
     batch = wl.make_batch(w, seed=seed, device="cuda")
     nb = {k: (v.cpu().numpy() if isinstance(v, torch.Tensor) and v.dtype != torch.bfloat16 else v)
           for k, v in batch.items() if k not in ("hidden", "W")}
     ref_sel = parity.oracle_selection(w, nb, seed, 0)
-    st = parity.gpu_step(w, batch, seed, 0)
+    st = parity.gpu_step(w, batch, seed, 0, fused=fused)
     parity.check_selection(st, ref_sel, w)
     assert st.status() == 0
     n = ref_sel["n_sel"]
@@ -102,6 +102,15 @@ def test_qwen3_0p6b_full():
 def test_qwen3_8b_full():
     n = _full_size_case("qwen3_8b")
     assert n > 100000
+
+
+def test_qwen3_8b_full_single_pass():
+    n = _full_size_case("qwen3_8b", fused=True)
+    assert n > 100000
+
+
+def test_qwen3_0p6b_full_single_pass():
+    _full_size_case("qwen3_0p6b", fused=True)
 
 
 def test_qwen3_8b_sweep_points():

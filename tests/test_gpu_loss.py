@@ -120,3 +120,66 @@ def test_unsupported_shapes_are_rejected():
     tiny_ws = nat.alloc_workspace(256, "cuda")
     with pytest.raises(nat.NatError):
         nat.nat_policy_loss_fwd(p, t, t, t, t, t, t, t, t, t, t, 4096, t, t, t, tiny_ws)
+
+
+# ---- single-pass route: nat_policy_loss_fwd_bwd ------------------------------------
+@pytest.mark.parametrize("name", ["tiny", "mid", "twin_0p6b", "twin_8b"])
+def test_fused_matches_oracle(name):
+    parity.run_case(wl.WORKLOADS[name], seed=0, fused=True)
+
+
+def test_fused_variants():
+    mid = wl.WORKLOADS["mid"]
+    parity.run_case(wl.variant(mid, sel_mode="rpc", min_cut=5), seed=0, fused=True)
+    out, _ = parity.run_case(wl.variant(mid, w_scale=0.5, old_noise=0.3), seed=1, fused=True)
+    assert out["dH_dense_err"] <= parity.TOL_DENSE
+    parity.run_case(wl.variant(mid, d=320, V=3001, P=4, G=8, len_lo=60, len_hi=200, p=0.75),
+                    seed=3, fused=True)
+
+
+def _two_chunk_batch(spike):
+    """~10k selected rows (two row chunks).  With `spike`, vocabulary row 700 gets a logit
+    of 100 * h[0]; h[0] is zero in the first half of the stream, so only the second chunk
+    leaves the single-pass window."""
+    w = wl.variant(wl.WORKLOADS["mid"], d=64, V=1024, P=8, G=8, len_lo=250, len_hi=380, p=0.5)
+    batch = wl.make_batch(w, seed=6, device="cuda")
+    if spike:
+        half = batch["n_tot"] // 2
+        batch["hidden"][:half, 0] = 0
+        batch["W"][700, :] = 0
+        batch["W"][700, 0] = 100.0
+        noise = torch.randn(batch["n_tot"], device="cuda") * 0.05
+        batch["old_logp"] = wl.library_logp(batch["hidden"], batch["W"], batch["targets"]) + noise
+    return w, batch
+
+
+@pytest.mark.parametrize("spike", [False, True])
+def test_fused_two_chunks_and_window_fallback(spike):
+    w, batch = _two_chunk_batch(spike)
+    nb = wl.to_numpy(batch)
+    ref_sel = parity.oracle_selection(w, nb, 6, 0)
+    assert 8192 < ref_sel["n_sel"] < 16384
+    st = parity.gpu_step(w, batch, 6, 0, fused=True)
+    parity.check_selection(st, ref_sel, w)
+    parity.check_loss(st, ref_sel, nb, w)
+    assert bool(st.status() & nat.NAT_DEV_FALLBACK) == spike
+    # the two routes agree with each other as well
+    st2 = parity.gpu_step(w, batch, 6, 0, fused=False)
+    n = ref_sel["n_sel"]
+    assert parity.rel_fro(st.dW.cpu().numpy(), st2.dW.cpu().numpy()) < 1e-2
+    assert float((st.logp[:n] - st2.logp[:n]).abs().max()) < 2 * parity.TOL_LOGP
+
+
+def test_fused_accumulate_and_dloss():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = parity.gpu_step(w, batch, 0, 0, fused=True)
+    base, baseH, loss = st.dW.clone(), st.dH.clone(), st.loss.clone()
+    dloss = torch.tensor([-2.0], device="cuda")
+    st.loss_fwd_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"],
+                    batch["cu_seqlens"], dloss=dloss, accumulate_dW=True)
+    torch.cuda.synchronize()
+    n = int(st.n_sel.item())
+    assert torch.equal(loss, st.loss)
+    assert parity.rel_fro(st.dW.cpu().numpy(), -base.cpu().numpy()) < 1e-2
+    assert parity.rel_fro(st.dH[:n].float().cpu().numpy(), -2 * baseH[:n].float().cpu().numpy()) < 1e-2
