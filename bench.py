@@ -3,7 +3,8 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
 A step is one pass of the whole path over one synthetic batch: advantages,
-selection, compaction, policy-loss forward and backward.  Rank 0 prints ONE
+selection, compaction, policy-loss forward and backward (by default through the
+single-pass call nat_policy_loss_fwd_bwd; --route two times the separate calls).  Rank 0 prints ONE
 JSON line.  `value` is selected tokens per second with inputs resident in HBM;
 `e2e` is the same with the step's inputs copied from pinned host memory and the
 loss read back inside the timed region.  `--impl reference` times the fp64 CPU
@@ -151,6 +152,7 @@ def run_ours(args, w):
     import torch.distributed as dist
 
     from paper_2603_06619_b200 import build as _build
+    from paper_2603_06619_b200 import sharding
     from paper_2603_06619_b200 import workloads as wl
     from paper_2603_06619_b200.step import NatStep
 
@@ -168,7 +170,7 @@ def run_ours(args, w):
 
     # Responses are independent, so ranks take disjoint batches (weak scaling):
     # no collective sits on the data path.
-    seed = args.seed + rank
+    seed = sharding.rank_seed(args.seed, rank)
     batch = wl.make_batch(w, seed=seed, device=dev)
     n_tot = batch["n_tot"]
     dtype = torch.float32 if w.dtype == "f32" else torch.bfloat16
@@ -180,8 +182,7 @@ def run_ours(args, w):
         st.grpo_adv(b["rewards"])
         st.select(cu, offset=offset, **sel)
         st.compact(cu)
-        st.loss_fwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
-        st.loss_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
+        st.loss_fwd_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -189,19 +190,25 @@ def run_ours(args, w):
             dist.barrier()
             torch.cuda.synchronize()
 
+    def step_two_pass(b, offset):
+        st.grpo_adv(b["rewards"])
+        st.select(cu, offset=offset, **sel)
+        st.compact(cu)
+        st.loss_fwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
+        st.loss_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
+
+    main_step = step if args.route == "single" else step_two_pass
     for i in range(args.warmup):
-        step(batch, i)
+        main_step(batch, i)
     sync_all()
-    if st.status() != 0:
+    if st.status() & ~4:
         raise RuntimeError(f"device status {st.status()} after warm-up")
 
+    # ---- device-resident timing of the whole step; the loss call bracketed by events
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-
-    # ---- device-resident timing; forward and backward bracketed separately
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    n_sel_total = 0
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     sync_all()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
@@ -212,22 +219,41 @@ def run_ours(args, w):
         st.select(cu, offset=off, **sel)
         st.compact(cu)
         ev[i][0].record()
-        st.loss_fwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
-        ev[i][1].record()
-        st.loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+        if args.route == "single":
+            st.loss_fwd_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+            ev[i][1].record()
+        else:
+            st.loss_fwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+            ev[i][1].record()
+            st.loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
         ev[i][2].record()
     t_end.record()
     sync_all()
+    clocks = sampler.stop() if rank == 0 else None
     elapsed_ms = t_begin.elapsed_time(t_end)
-    fwd_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
-    bwd_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    loss_call_ms = statistics.mean(e[0].elapsed_time(e[2]) for e in ev)
+    first_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    status = st.status()
+    loss_val = float(st.loss.item())
     # selected tokens per step: selection with offsets warmup..warmup+K-1 (replayed, untimed)
+    n_sel_total = 0
     for i in range(args.steps):
         st.select(cu, offset=args.warmup + i, **sel)
         st.compact(cu)
         n_sel_total += int(st.n_sel.item())
-    status = st.status()
-    loss_val = float(st.loss.item())
+
+    # ---- the other route, for the record (same batch, same offsets, 1 warm-up)
+    other = step_two_pass if args.route == "single" else step
+    other(batch, 0)
+    sync_all()
+    o_begin = torch.cuda.Event(enable_timing=True)
+    o_end = torch.cuda.Event(enable_timing=True)
+    o_begin.record()
+    for i in range(args.steps):
+        other(batch, args.warmup + i)
+    o_end.record()
+    sync_all()
+    other_ms = o_begin.elapsed_time(o_end)
 
     # ---- end to end: the step's inputs come from pinned host memory
     host = {k: batch[k].cpu().pin_memory() for k in ("hidden", "targets", "old_logp", "rewards")}
@@ -239,7 +265,7 @@ def run_ours(args, w):
         for k in host:
             dev_in[k].copy_(host[k], non_blocking=True)
         b = dict(dev_in, W=batch["W"])
-        step(b, offset)
+        main_step(b, offset)
         loss_host.copy_(st.loss, non_blocking=True)
 
     e2e_step(0)
@@ -252,16 +278,10 @@ def run_ours(args, w):
     e_end.record()
     sync_all()
     e2e_ms = e_begin.elapsed_time(e_end)
-    clocks = sampler.stop() if rank == 0 else None
 
     # ---- max over ranks, totals over ranks
-    stats = torch.tensor([elapsed_ms, e2e_ms, fwd_ms, bwd_ms], dtype=torch.float64, device=dev)
-    total = torch.tensor([float(n_sel_total)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-        dist.all_reduce(total, op=dist.ReduceOp.SUM)
-    elapsed_ms, e2e_ms, fwd_ms, bwd_ms = (float(x) for x in stats.tolist())
-    n_all = float(total.item())
+    (elapsed_ms, e2e_ms, loss_call_ms, first_ms, other_ms), n_all = sharding.aggregate_timing(
+        [elapsed_ms, e2e_ms, loss_call_ms, first_ms, other_ms], n_sel_total, device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -270,15 +290,26 @@ def run_ours(args, w):
     peaks, peak_kind = load_peaks()
     n_step = n_sel_total / args.steps              # this rank's selected tokens per step
     dV = float(w.d) * float(w.V)
-    # The step runs for seconds under the power cap, so the sustained tensor
-    # peak is the denominator; the burst figure is reported beside it.
+    # The step runs for most of a second under the power cap, so the sustained tensor
+    # peak is the roofline's denominator; the burst figure is reported beside it.
     peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-    bwd_tflops = 4.0 * n_step * dV / (bwd_ms * 1e-3) / 1e12
-    fwd_tflops = 2.0 * n_step * dV / (fwd_ms * 1e-3) / 1e12
     step_ms = elapsed_ms / args.steps
+    counted = 6.0 * n_step * dV
+    executed = counted if args.route == "single" else 8.0 * n_step * dV
+    call_tflops = counted / (loss_call_ms * 1e-3) / 1e12
+    step_tflops = counted / (step_ms * 1e-3) / 1e12
     cap_pad = (n_tot + 127) // 128 * 128
     n_chunks = (cap_pad + min(cap_pad, 8192) - 1) // min(cap_pad, 8192)
-    launches = 1 + (1 if w.sel_mode == "urs" else 2) + 3 + 4 + (3 + 3 * n_chunks)
+    sel_launches = 1 + (1 if w.sel_mode == "urs" else 2) + 3
+    if w.dtype == "f32":
+        launches = sel_launches + 2 + 3
+    elif args.route == "single":
+        launches = sel_launches + 2 + 9 * n_chunks + 3
+    else:
+        launches = sel_launches + 4 + (3 + 3 * n_chunks)
+    kernel = ("nat_tc_kernel<kE|kDh|kDw> (the launches inside nat_policy_loss_fwd_bwd)"
+              if args.route == "single" else
+              "nat_tc_kernel<kFwd|kDz|kDh|kDw> (nat_policy_loss_fwd + nat_policy_loss_bwd)")
 
     line = {
         "metric": METRIC, "value": n_all / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -287,30 +318,36 @@ def run_ours(args, w):
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": w.name, "P": w.P, "G": w.G, "d": w.d, "V": w.V,
                    "selection": w.sel_mode, "p": w.p, "min_cut": w.min_cut,
+                   "route": ("single pass (nat_policy_loss_fwd_bwd)" if args.route == "single"
+                             else "two pass (nat_policy_loss_fwd, nat_policy_loss_bwd)"),
                    "n_tot_per_gpu": n_tot, "n_sel_per_step_per_gpu": n_step,
                    "l2": "inputs larger than L2 (hidden and W_lm are GBs); no flush needed",
                    "parallelism": f"dp{world} (independent batches, no collective)"},
-        "tflops_counted": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12,
-        "tflops_executed": 8.0 * n_step * dV / (step_ms * 1e-3) / 1e12,
+        "tflops_counted": step_tflops,
+        "tflops_executed": executed / (step_ms * 1e-3) / 1e12,
         "frac_of_peak_counted": {
-            "burst": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12 / float(peaks["bf16_tflops"]),
-            "sustained": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12 / peak,
-            "datasheet_2250": 6.0 * n_step * dV / (step_ms * 1e-3) / 1e12 / 2250.0},
-        "fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "loss": loss_val, "device_status": status,
+            "burst": step_tflops / float(peaks["bf16_tflops"]),
+            "sustained": step_tflops / peak,
+            "datasheet_2250": step_tflops / 2250.0},
+        "loss_call_ms": loss_call_ms, "loss": loss_val, "device_status": status,
+        "other_route": {"route": "two pass" if args.route == "single" else "single pass",
+                        "ms_per_step": other_ms / args.steps,
+                        "tflops_counted": counted / (other_ms / args.steps * 1e-3) / 1e12},
         "roofline": {
-            "kernel": "nat_tc_kernel<kDz|kDh|kDw> (the launches inside nat_policy_loss_bwd)",
-            "bound": "tensor", "achieved": bwd_tflops, "peak": peak, "unit": "TFLOP/s",
-            "frac": bwd_tflops / peak, "peak_source": f"{peak_kind} bf16_tflops_sustained",
-            "flops": "counted 4*N_sel*d*V per backward call (6*N_sel*d*V executed with the recompute)",
+            "kernel": kernel, "bound": "tensor", "achieved": call_tflops, "peak": peak,
+            "unit": "TFLOP/s", "frac": call_tflops / peak,
+            "peak_source": f"{peak_kind} bf16_tflops_sustained (of measured)"
+            if peak_kind == "measured" else "fallback (of fallback)",
+            "flops": "counted 6*N_sel*d*V per step (2 forward + 4 backward), divided by the "
+                     "event-timed duration of the loss call(s), small kernels included",
             "traffic": None},
-        "roofline_fwd": {
-            "kernel": "nat_tc_kernel<kFwd>", "bound": "tensor", "achieved": fwd_tflops,
-            "peak": peak, "unit": "TFLOP/s", "frac": fwd_tflops / peak, "traffic": None},
         "e2e": {"value": n_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": 4, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": launches * args.steps,
         "clocks": clocks,
     }
+    if args.route == "two":
+        line["fwd_ms"], line["bwd_ms"] = first_ms, loss_call_ms - first_ms
     if not args.no_cpu_baseline and world == 1:
         rate, secs, n, _ = oracle_sample_rate(w, seed=0, rows=args.ref_rows)
         line["cpu_baseline"] = {
@@ -332,6 +369,8 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--route", default="single", choices=["single", "two"],
+                    help="single: nat_policy_loss_fwd_bwd; two: forward then backward calls")
     args = ap.parse_args()
     from paper_2603_06619_b200 import workloads as wl
     w = wl.WORKLOADS[args.workload]
