@@ -29,6 +29,7 @@
 // Every mbarrier wait is bounded; a wait that runs out raises the block's
 // abort flag and NAT_DEV_TIMEOUT in the workspace's status word.
 #include <cuda_bf16.h>
+#include <cstdlib>
 
 #include "nat_tc.cuh"
 #include "nat_token.cuh"
@@ -37,17 +38,14 @@ namespace nat {
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages = 4;
 constexpr int kABytes = BM * BK * 2;               // 16 KB
-constexpr int kBBytes = BN * BK * 2;               // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;     // 48 KB
 constexpr int kBoxBytes = 64 * 64 * 2;             // one 64x64 box of an MN-major operand
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;                     // two 256-column accumulators
 constexpr int kGroupRows = 16;                     // row blocks that share a vocabulary sweep
 constexpr int kTilesPerSplit = 16;                 // vocabulary tiles per work unit
 constexpr int kChunkRows = 8192;                   // rows of the dZ scratch
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr int kRowPad = 256;                       // compact rows are padded to a pair's M extent
 
 enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3, kE = 4 };
 
@@ -97,8 +95,9 @@ struct Shape {
   int nblocks;  // N blocks (kDh, kDw) or vocabulary tiles (kFwd, kDz)
 };
 
-template <int MODE>
+template <int MODE, int CTAS>
 __device__ __forceinline__ Shape make_shape(const TcParams& p) {
+  constexpr int BMU = BM * CTAS;  // rows of the accumulator's M dimension per work unit
   Shape s;
   int n = *p.n_sel;
   n = n < p.cap ? n : p.cap;
@@ -107,17 +106,17 @@ __device__ __forceinline__ Shape make_shape(const TcParams& p) {
   if (p.flag != nullptr && ((*p.flag != 0) ? 1 : 0) != p.run_if) rows = 0;
   s.rows = rows;
   if (MODE == kFwd || MODE == kDz || MODE == kE) {
-    s.mblocks = (rows + BM - 1) / BM;
+    s.mblocks = (rows + BMU - 1) / BMU;
     s.nblocks = (p.V + BN - 1) / BN;
     s.n_units = s.mblocks * p.n_splits;
     s.kb = p.d / BK;
   } else if (MODE == kDh) {
-    s.mblocks = (rows + BM - 1) / BM;
+    s.mblocks = (rows + BMU - 1) / BMU;
     s.nblocks = (p.d + BN - 1) / BN;
     s.n_units = s.mblocks * s.nblocks;
     s.kb = (p.V + BK - 1) / BK;
   } else {
-    s.mblocks = (p.V + BM - 1) / BM;
+    s.mblocks = (p.V + BMU - 1) / BMU;
     s.nblocks = (p.d + BN - 1) / BN;
     s.kb = (rows + BK - 1) / BK;
     s.n_units = rows > 0 ? s.mblocks * s.nblocks : 0;
@@ -126,19 +125,20 @@ __device__ __forceinline__ Shape make_shape(const TcParams& p) {
 }
 
 // Units are ordered so that CTAs running side by side share operands in L2:
-// kFwd/kDz take groups of kGroupRows row blocks and, inside a group, walk the
-// vocabulary splits with the row block varying fastest.
-template <int MODE>
+// kFwd/kDz/kE take groups of row blocks (kGroupRows x 128 rows) and, inside a
+// group, walk the vocabulary splits with the row block varying fastest.
+template <int MODE, int CTAS>
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Shape& s, int u) {
+  constexpr int kGroup = kGroupRows / CTAS;
   Unit w;
   if (MODE == kFwd || MODE == kDz || MODE == kE) {
-    const int per_group = kGroupRows * p.n_splits;
+    const int per_group = kGroup * p.n_splits;
     const int grp = u / per_group;
     const int rem = u - grp * per_group;
-    int rows_in_group = s.mblocks - grp * kGroupRows;
-    rows_in_group = rows_in_group < kGroupRows ? rows_in_group : kGroupRows;
+    int rows_in_group = s.mblocks - grp * kGroup;
+    rows_in_group = rows_in_group < kGroup ? rows_in_group : kGroup;
     w.sp = rem / rows_in_group;
-    w.mb = grp * kGroupRows + (rem - w.sp * rows_in_group);
+    w.mb = grp * kGroup + (rem - w.sp * rows_in_group);
     w.nt_lo = (int)(((long long)w.sp * s.nblocks) / p.n_splits);
     w.nt_hi = (int)(((long long)(w.sp + 1) * s.nblocks) / p.n_splits);
   } else {
@@ -163,35 +163,53 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
-template <int MODE>
+// Shared-memory ring: CTAS = 1: 4 stages of (A 128x64 + B 256x64) = 48 KB;
+// CTAS = 2: each CTA of the pair holds its 128 rows of A and its 128-row half
+// of B, 32 KB per stage, 6 stages.
+template <int CTAS>
+struct Ring {
+  static constexpr int kBRows = BN / CTAS;
+  static constexpr int kBBytes = kBRows * BK * 2;
+  static constexpr int kStage = kABytes + kBBytes;
+  static constexpr int kNum = CTAS == 1 ? 4 : 6;
+  static constexpr size_t kSmem = (size_t)kNum * kStage + 1024 /*alignment*/ + 256 /*barriers*/;
+};
+
+template <int MODE, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
               const TcParams p) {
+  using R = Ring<CTAS>;
+  constexpr int kNS = R::kNum;
+  constexpr int BMU = BM * CTAS;
   constexpr bool kAmn = (MODE == kDw);
   constexpr bool kBmn = (MODE == kDh || MODE == kDw);
-  constexpr uint32_t kIdesc = tc::instr_desc_bf16(BM, BN, kAmn ? 1 : 0, kBmn ? 1 : 0);
+  constexpr uint32_t kIdesc = tc::instr_desc_bf16(BMU, BN, kAmn ? 1 : 0, kBmn ? 1 : 0);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);
-  uint64_t* full_bar = bars;                    // [kStages]
-  uint64_t* empty_bar = bars + kStages;         // [kStages]
-  uint64_t* tfull_bar = bars + 2 * kStages;     // [2]
-  uint64_t* tempty_bar = bars + 2 * kStages + 2;  // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kNS * R::kStage);
+  uint64_t* full_bar = bars;                   // [kNS]   (CTAS = 2: the even CTA's are used)
+  uint64_t* empty_bar = bars + kNS;            // [kNS]
+  uint64_t* tfull_bar = bars + 2 * kNS;        // [2]
+  uint64_t* tempty_bar = bars + 2 * kNS + 2;   // [2]     (CTAS = 2: the even CTA's are used)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kNS + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const int rank = CTAS == 2 ? (int)(tc::cluster_ctarank() & 1u) : 0;
+  const int unit0 = blockIdx.x / CTAS;
+  const int unit_stride = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kNS; ++s) {
       tc::mbar_init(&full_bar[s], 1);
       tc::mbar_init(&empty_bar[s], 1);
     }
     for (int a = 0; a < 2; ++a) {
       tc::mbar_init(&tfull_bar[a], 1);
-      tc::mbar_init(&tempty_bar[a], 4);
+      tc::mbar_init(&tempty_bar[a], 4 * CTAS);
     }
     *abort_flag = 0u;
     tc::fence_barrier_init();
@@ -200,61 +218,78 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     tc::prefetch_tensormap(&mapB);
   }
   if (warp == 1) {
-    tc::tmem_alloc(tmem_slot, kTmemCols);
-    tc::tmem_relinquish();
+    if (CTAS == 2) {
+      tc::tmem_alloc_pair(tmem_slot, kTmemCols);
+      tc::tmem_relinquish_pair();
+    } else {
+      tc::tmem_alloc(tmem_slot, kTmemCols);
+      tc::tmem_relinquish();
+    }
   }
   tc::fence_before_sync();
   __syncthreads();
+  if (CTAS == 2) tc::cluster_sync_all();  // the peer's barriers exist before anyone signals them
   tc::fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  const Shape shape = make_shape<MODE>(p);
+  const Shape shape = make_shape<MODE, CTAS>(p);
 
   if (warp == 0) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < shape.n_units; u += gridDim.x) {
-        const Unit w = decode_unit<MODE>(p, shape, u);
+      for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
+        const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
         for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt) {
           for (int kb = 0; kb < shape.kb; ++kb, ++it) {
-            const int s = it % kStages;
-            const uint32_t ph = (it / kStages) & 1u;
+            const int s = it % kNS;
+            const uint32_t ph = (it / kNS) & 1u;
             if (!tc::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-            uint8_t* a_dst = smem + (size_t)s * kStageBytes;
+            uint8_t* a_dst = smem + (size_t)s * R::kStage;
             uint8_t* b_dst = a_dst + kABytes;
-            tc::mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
+            // CTAS = 2: both CTAs' loads count on the even CTA's barrier, which its
+            // own producer arms with the bytes of the whole pair.
+            const uint32_t bar = CTAS == 2 ? tc::map_to_cta(tc::smem_u32(&full_bar[s]), 0)
+                                           : tc::smem_u32(&full_bar[s]);
+            if (rank == 0) tc::mbar_arrive_expect_tx(&full_bar[s], R::kStage * CTAS);
+            auto load = [&](void* dst, const CUtensorMap* map, int x, int y) {
+              if (CTAS == 2) tc::tma_load_2d_pair(dst, map, bar, x, y);
+              else tc::tma_load_2d(dst, map, &full_bar[s], x, y);
+            };
+            const int m0 = w.mb * BMU + rank * BM;            // this CTA's rows of A / D
+            const int n0 = nt * BN + rank * R::kBRows;        // this CTA's rows of B
             if (MODE == kFwd || MODE == kDz || MODE == kE) {
-              tc::tma_load_2d(a_dst, &mapA, &full_bar[s], kb * BK, p.row0 + w.mb * BM);
-              tc::tma_load_2d(b_dst, &mapB, &full_bar[s], kb * BK, nt * BN);
+              load(a_dst, &mapA, kb * BK, p.row0 + m0);
+              load(b_dst, &mapB, kb * BK, n0);
             } else if (MODE == kDh) {
-              tc::tma_load_2d(a_dst, &mapA, &full_bar[s], kb * BK, w.mb * BM);
+              load(a_dst, &mapA, kb * BK, m0);
 #pragma unroll
-              for (int j = 0; j < BN / 64; ++j)
-                tc::tma_load_2d(b_dst + j * kBoxBytes, &mapB, &full_bar[s], nt * BN + j * 64,
-                                kb * BK);
+              for (int j = 0; j < R::kBRows / 64; ++j)
+                load(b_dst + j * kBoxBytes, &mapB, n0 + j * 64, kb * BK);
             } else {
 #pragma unroll
               for (int j = 0; j < BM / 64; ++j)
-                tc::tma_load_2d(a_dst + j * kBoxBytes, &mapA, &full_bar[s], w.mb * BM + j * 64,
-                                kb * BK);
+                load(a_dst + j * kBoxBytes, &mapA, m0 + j * 64, kb * BK);
 #pragma unroll
-              for (int j = 0; j < BN / 64; ++j)
-                tc::tma_load_2d(b_dst + j * kBoxBytes, &mapB, &full_bar[s], nt * BN + j * 64,
-                                p.b_row0 + kb * BK);
+              for (int j = 0; j < R::kBRows / 64; ++j)
+                load(b_dst + j * kBoxBytes, &mapB, n0 + j * 64, p.b_row0 + kb * BK);
             }
           }
         }
       }
-      if (!ok) {
-        // Loads already issued still complete on their own; give them a
-        // bounded chance to land before the block's shared memory is released.
-        const uint32_t pending = it < (uint32_t)kStages ? it : (uint32_t)kStages;
-        for (uint32_t j = 0; j < pending; ++j) {
-          const uint32_t jt = it - 1 - j;
+      // Tail: wait until every stage this thread filled has been released, so that no
+      // arrival (from this CTA's MMA or the peer's) targets this CTA after it has left,
+      // and no load is still writing its shared memory.  Bounded like every wait.
+      const uint32_t pending = it < (uint32_t)kNS ? it : (uint32_t)kNS;
+      for (uint32_t j = 0; j < pending; ++j) {
+        const uint32_t jt = it - 1 - j;
+        if (ok) {
+          if (!tc::mbar_wait(&empty_bar[jt % kNS], (jt / kNS) & 1u, abort_flag)) ok = false;
+        }
+        if (!ok && CTAS == 1) {
           const uint64_t t0 = tc::global_timer_ns();
-          while (!tc::mbar_try_wait(&full_bar[jt % kStages], (jt / kStages) & 1u)) {
+          while (!tc::mbar_try_wait(&full_bar[jt % kNS], (jt / kNS) & 1u)) {
             if (tc::global_timer_ns() - t0 > 100000000ull) break;
           }
         }
@@ -262,12 +297,12 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------ MMA issuer (even CTA of a pair)
+    if (lane == 0 && rank == 0) {
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int u = blockIdx.x; ok && u < shape.n_units; u += gridDim.x) {
-        const Unit w = decode_unit<MODE>(p, shape, u);
+      for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
+        const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
         for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt, ++tcount) {
           const uint32_t acc = tcount & 1u;
           const uint32_t aph = (tcount >> 1) & 1u;
@@ -275,11 +310,11 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
           tc::fence_after_sync();
           const uint32_t d_tmem = tmem_base + acc * BN;
           for (int kb = 0; kb < shape.kb; ++kb, ++it) {
-            const int s = it % kStages;
-            const uint32_t ph = (it / kStages) & 1u;
+            const int s = it % kNS;
+            const uint32_t ph = (it / kNS) & 1u;
             if (!tc::mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
             tc::fence_after_sync();
-            const uint32_t a_base = tc::smem_u32(smem + (size_t)s * kStageBytes);
+            const uint32_t a_base = tc::smem_u32(smem + (size_t)s * R::kStage);
             const uint32_t b_base = a_base + kABytes;
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk) {
@@ -294,11 +329,16 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
               const uint64_t bdesc =
                   kBmn ? tc::smem_desc_sw128(b_base + kk * 2048, kBoxBytes, 1024)
                        : tc::smem_desc_sw128(b_base + kk * 32, 16, 1024);
-              tc::umma_bf16(d_tmem, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+              if (CTAS == 2) tc::umma_bf16_pair(d_tmem, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+              else tc::umma_bf16(d_tmem, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
             }
-            tc::umma_commit(&empty_bar[s]);
+            if (CTAS == 2) tc::umma_commit_pair(&empty_bar[s], 3);
+            else tc::umma_commit(&empty_bar[s]);
           }
-          if (ok) tc::umma_commit(&tfull_bar[acc]);
+          if (ok) {
+            if (CTAS == 2) tc::umma_commit_pair(&tfull_bar[acc], 3);
+            else tc::umma_commit(&tfull_bar[acc]);
+          }
         }
       }
     }
@@ -309,9 +349,9 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     const int n_valid = p.row0 + shape.rows;  // compact rows below this are real tokens
     uint32_t tcount = 0;
     bool ok = true;
-    for (int u = blockIdx.x; ok && u < shape.n_units; u += gridDim.x) {
-      const Unit w = decode_unit<MODE>(p, shape, u);
-      const int lrow = w.mb * BM + q * 32 + lane;  // row inside this launch's M range
+    for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
+      const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
+      const int lrow = w.mb * BMU + rank * BM + q * 32 + lane;  // row inside this launch's M range
       // per-unit row state
       float m_run = -INFINITY, s_run = 0.f, zt_val = 0.f;
       bool zt_found = false;
@@ -449,7 +489,10 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         }
         tc::fence_before_sync();
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&tempty_bar[acc]);
+        if (lane == 0) {
+          if (CTAS == 2) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&tempty_bar[acc]), 0));
+          else tc::mbar_arrive(&tempty_bar[acc]);
+        }
       }
       if (MODE == kFwd && ok && row_ok) {
         const int k = p.row0 + lrow;
@@ -469,9 +512,11 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
   tc::fence_before_sync();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag != 0u) atomicOr(p.status, NAT_DEV_TIMEOUT);
+  if (CTAS == 2) tc::cluster_sync_all();  // the pair leaves together
   if (warp == 1) {
     tc::fence_after_sync();
-    tc::tmem_dealloc(tmem_base, kTmemCols);
+    if (CTAS == 2) tc::tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tc::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -557,7 +602,7 @@ __global__ void fused_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_
   const int vec = d / 8;
   for (int r = blockIdx.x; r < chunk_rows; r += gridDim.x) {
     const int k = row0 + r;
-    if (k >= n && r >= ((n - row0 + BM - 1) / BM) * BM) break;  // beyond the tiles in use
+    if (k >= n && r >= ((n - row0 + kRowPad - 1) / kRowPad) * kRowPad) break;  // beyond the tiles in use
     __syncthreads();
     if (threadIdx.x == 0) {
       float cv = 0.f;
@@ -636,7 +681,7 @@ struct Layout {
 Layout make_layout(const nat_loss_params& p, int64_t cap) {
   Layout L;
   const int64_t c1 = cap > 0 ? cap : 1;
-  L.cap_pad = (int)((c1 + BM - 1) / BM * BM);
+  L.cap_pad = (int)((c1 + kRowPad - 1) / kRowPad * kRowPad);
   L.n_tiles = (p.V + BN - 1) / BN;
   L.n_splits = (L.n_tiles + kTilesPerSplit - 1) / kTilesPerSplit;
   L.chunk_rows = L.cap_pad < kChunkRows ? L.cap_pad : kChunkRows;
@@ -714,23 +759,79 @@ int sm_count(int* out) {
   return NAT_OK;
 }
 
-template <int MODE>
-int launch_tc(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, int max_units,
-              cudaStream_t stream) {
+
+// CTA pairs (cta_group::2) halve each CTA's share of the B operand and are used whenever
+// the device can co-schedule 2-CTA clusters of this kernel on (nearly) all of its SMs;
+// otherwise (e.g. a partitioned GPU) the single-CTA kernels run.
+int pair_slots() {
+  static int slots = -1;
+  if (slots < 0) {
+    slots = 0;
+    int sms = 0;
+    if (sm_count(&sms) == NAT_OK &&
+        cudaFuncSetAttribute(nat_tc_kernel<kFwd, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Ring<2>::kSmem) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)sms, 1, 1);
+      cfg.blockDim = dim3(kThreads, 1, 1);
+      cfg.dynamicSmemBytes = Ring<2>::kSmem;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      int clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&clusters, nat_tc_kernel<kFwd, 2>, &cfg) == cudaSuccess &&
+          clusters * 2 * 10 >= sms * 9)
+        slots = clusters;
+    }
+    (void)cudaGetLastError();
+  }
+  return slots;
+}
+
+template <int MODE, int CTAS>
+int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, int max_units,
+                   cudaStream_t stream) {
   static bool configured = false;
   if (!configured) {
-    NAT_CUDA(cudaFuncSetAttribute(nat_tc_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)kSmemBytes));
+    NAT_CUDA(cudaFuncSetAttribute(nat_tc_kernel<MODE, CTAS>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)Ring<CTAS>::kSmem));
     configured = true;
   }
   int sms = 0;
   int s = sm_count(&sms);
   if (s != NAT_OK) return s;
-  const int grid = max_units < sms ? max_units : sms;
-  if (grid <= 0) return NAT_OK;
-  nat_tc_kernel<MODE><<<grid, kThreads, kSmemBytes, stream>>>(a, b, p);
-  NAT_LAUNCH_CHECK("nat_tc_kernel");
+  const int slots = CTAS == 2 ? pair_slots() : sms;
+  const int groups = max_units < slots ? max_units : slots;
+  if (groups <= 0) return NAT_OK;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(groups * CTAS), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = Ring<CTAS>::kSmem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  NAT_CUDA(cudaLaunchKernelEx(&cfg, nat_tc_kernel<MODE, CTAS>, a, b, p));
   return NAT_OK;
+}
+
+// `units128`: number of work units when the M dimension is cut into 128-row blocks
+// (m_blocks128 * per_block); a pair covers two such blocks per unit.
+template <int MODE>
+int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2,
+              const TcParams& p, int m_blocks128, int per_block, cudaStream_t stream) {
+  if (pair_slots() > 0)
+    return launch_tc_impl<MODE, 2>(a, b2, p, ((m_blocks128 + 1) / 2) * per_block, stream);
+  return launch_tc_impl<MODE, 1>(a, b1, p, m_blocks128 * per_block, stream);
 }
 
 TokenCtx make_ctx(const LossArgs& a) {
@@ -815,7 +916,7 @@ int gather(const LossArgs& a, const Layout& L, const Ws& w) {
 }
 
 struct Maps {
-  CUtensorMap hcK, wK, dzK, wMn, dzMn, hcMn, hsMn;
+  CUtensorMap hcK, wK, wK2, dzK, wMn, dzMn, hcMn, hsMn;  // wK2: 128-row boxes for CTA pairs
 };
 
 int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
@@ -823,6 +924,7 @@ int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
   const uint64_t dpitch = (uint64_t)a.p.d * 2, zpitch = (uint64_t)L.ldz * 2;
   if ((s = make_map(&m->hcK, w.hc, a.p.d, L.cap_pad, dpitch, BK, BM)) != NAT_OK) return s;
   if ((s = make_map(&m->wK, a.W, a.p.d, a.p.V, dpitch, BK, BN)) != NAT_OK) return s;
+  if ((s = make_map(&m->wK2, a.W, a.p.d, a.p.V, dpitch, BK, BN / 2)) != NAT_OK) return s;
   if ((s = make_map(&m->dzK, w.dz, a.p.V, L.chunk_rows, zpitch, BK, BM)) != NAT_OK) return s;
   if ((s = make_map(&m->wMn, a.W, a.p.d, a.p.V, dpitch, 64, BK)) != NAT_OK) return s;
   if ((s = make_map(&m->dzMn, w.dz, a.p.V, L.chunk_rows, zpitch, 64, BK)) != NAT_OK) return s;
@@ -849,9 +951,9 @@ int launch_two_pass_chunk(const LossArgs& a, const Layout& L, const Ws& w, const
   p.run_if = 1;
   const int mb = L.chunk_rows / BM;
   const int nb_d = (a.p.d + BN - 1) / BN;
-  if ((s = launch_tc<kDz>(m.hcK, m.wK, p, mb * L.n_splits, a.stream)) != NAT_OK) return s;
-  if ((s = launch_tc<kDh>(m.dzK, m.wMn, p, mb * nb_d, a.stream)) != NAT_OK) return s;
-  return launch_tc<kDw>(m.dzMn, m.hcMn, p, ((a.p.V + BM - 1) / BM) * nb_d, a.stream);
+  if ((s = launch_tc<kDz>(m.hcK, m.wK, m.wK2, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
+  if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, p, mb, nb_d, a.stream)) != NAT_OK) return s;
+  return launch_tc<kDw>(m.dzMn, m.hcMn, m.hcMn, p, (a.p.V + BM - 1) / BM, nb_d, a.stream);
 }
 
 int launch_onehot(const LossArgs& a, const Ws& w) {
@@ -877,11 +979,11 @@ int loss_bf16_fwd(const LossArgs& a) {
   const TokenCtx c = make_ctx(a);
   if (a.cap > 0) {
     if ((s = gather(a, L, w)) != NAT_OK) return s;
-    CUtensorMap mapA, mapB;
-    if ((s = make_map(&mapA, w.hc, a.p.d, L.cap_pad, (uint64_t)a.p.d * 2, BK, BM)) != NAT_OK) return s;
-    if ((s = make_map(&mapB, a.W, a.p.d, a.p.V, (uint64_t)a.p.d * 2, BK, BN)) != NAT_OK) return s;
+    Maps m;
+    if ((s = make_maps(a, L, w, &m)) != NAT_OK) return s;
     const TcParams p = base_params(a, L, w);
-    if ((s = launch_tc<kFwd>(mapA, mapB, p, (L.cap_pad / BM) * L.n_splits, a.stream)) != NAT_OK)
+    if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, p, L.cap_pad / BM, L.n_splits, a.stream)) !=
+        NAT_OK)
       return s;
     fwd_finalize_kernel<<<finalize_grid((int)a.cap), 256, 0, a.stream>>>(
         c, a.n_sel, (int)a.cap, 0, L.cap_pad, L.n_splits, L.cap_pad, w.pm, w.ps, w.zt, a.logp,
@@ -934,7 +1036,8 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.V = a.p.V < BN ? a.p.V : BN;
       p.n_splits = 1;
       p.part_m = w.mref;
-      if ((s = launch_tc<kFwd>(m.hcK, m.wK, p, L.cap_pad / BM, a.stream)) != NAT_OK) return s;
+      if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, p, L.cap_pad / BM, 1, a.stream)) != NAT_OK)
+        return s;
     }
     for (int ci = 0; ci < L.n_chunks; ++ci) {
       const int row0 = ci * L.chunk_rows;
@@ -943,7 +1046,7 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.row0 = row0;
       p.chunk_rows = L.chunk_rows;
       p.ovf = ovf;
-      if ((s = launch_tc<kE>(m.hcK, m.wK, p, mb * L.n_splits, a.stream)) != NAT_OK) return s;
+      if ((s = launch_tc<kE>(m.hcK, m.wK, m.wK2, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
       fused_finalize_kernel<<<L.chunk_rows < 2048 ? L.chunk_rows : 2048, 128, 0, a.stream>>>(
           c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_splits, L.cap_pad, w.mref, w.ps, w.zt,
           a.dloss, a.logp, a.lse, w.term, w.g, w.cs, w.hc, w.hs, a.p.d, ovf);
@@ -953,9 +1056,9 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.run_if = 0;
       p.row_scale = w.cs;
       p.b_row0 = 0;  // Hs is local to the chunk
-      if ((s = launch_tc<kDh>(m.dzK, m.wMn, p, mb * nb_d, a.stream)) != NAT_OK) return s;
-      if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, p, ((a.p.V + BM - 1) / BM) * nb_d, a.stream)) !=
-          NAT_OK)
+      if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, p, mb, nb_d, a.stream)) != NAT_OK) return s;
+      if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, m.hsMn, p, (a.p.V + BM - 1) / BM, nb_d,
+                              a.stream)) != NAT_OK)
         return s;
       // Predicated redo of the chunk by the two-pass kernels (no-ops unless *ovf != 0).
       TcParams pf = base_params(a, L, w);
@@ -963,7 +1066,8 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       pf.chunk_rows = L.chunk_rows;
       pf.flag = ovf;
       pf.run_if = 1;
-      if ((s = launch_tc<kFwd>(m.hcK, m.wK, pf, mb * L.n_splits, a.stream)) != NAT_OK) return s;
+      if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, pf, mb, L.n_splits, a.stream)) != NAT_OK)
+        return s;
       fwd_finalize_kernel<<<finalize_grid(L.chunk_rows), 256, 0, a.stream>>>(
           c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_splits, L.cap_pad, w.pm, w.ps, w.zt,
           a.logp, a.lse, w.term, w.g, a.dloss, ovf, 1);
