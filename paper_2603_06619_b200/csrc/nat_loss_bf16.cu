@@ -45,6 +45,7 @@ constexpr int kTmemCols = 512;                     // two 256-column accumulator
 constexpr int kGroupRows = 16;                     // row blocks that share a vocabulary sweep
 constexpr int kTilesPerSplit = 16;                 // vocabulary tiles per work unit
 constexpr int kChunkRows = 8192;                   // rows of the dZ scratch
+constexpr int kMaxPairs = 512;                     // progress marks (one per CTA or CTA pair)
 constexpr int kRowPad = 256;                       // compact rows are padded to a pair's M extent
 
 enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3, kE = 4 };
@@ -78,6 +79,8 @@ struct TcParams {
   const int32_t* flag;     // predicate: the launch does nothing unless
   int run_if;              //   (*flag != 0) == run_if   (flag == null: always runs)
   int32_t* ovf;            // kE: set to 1 when the window is exceeded
+  unsigned long long* progress;  // per-pair progress marks of the vocabulary sweeps
+  unsigned long long epoch;      // distinguishes this launch's marks from earlier ones
 };
 
 struct Unit {
@@ -242,6 +245,37 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
         const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
         for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt) {
+          if ((MODE == kFwd || MODE == kDz || MODE == kE) && rank == 0 && p.progress != nullptr) {
+            // Pacing.  The CTAs that sweep the same vocabulary split for different row
+            // blocks share every W tile through L2 only while they stay within a few
+            // tiles of each other; left alone they drift apart (nothing slows the one in
+            // front) and each W tile is then read from DRAM several times, which costs
+            // more power than the tensor cores can spare.  So each CTA publishes the tile
+            // it is starting and briefly holds back while a mate is more than a tile
+            // behind.  Purely advisory: the wait is short and bounded, and results do not
+            // depend on it.
+            constexpr int kGroup = kGroupRows / CTAS;
+            volatile unsigned long long* marks = p.progress;
+            const int j = nt - w.nt_lo;
+            const unsigned long long iter = (unsigned long long)((u - unit0) / unit_stride);
+            marks[unit0] = (p.epoch << 40) | (iter << 10) | (unsigned long long)j;
+            if (j > 0) {
+              const int per_group = kGroup * p.n_splits;
+              const int grp = u / per_group;
+              int mates = shape.mblocks - grp * kGroup;
+              mates = mates < kGroup ? mates : kGroup;
+              const int first = grp * per_group + w.sp * mates;
+              for (int r = 0; r < mates; ++r) {
+                const int um = first + r;
+                if (um == u) continue;
+                const unsigned long long want = (p.epoch << 40) |
+                                                ((unsigned long long)(um / unit_stride) << 10) |
+                                                (unsigned long long)(j - 1);
+                const int pm = um % unit_stride;
+                for (int spin = 0; spin < 64 && marks[pm] < want; ++spin) __nanosleep(100);
+              }
+            }
+          }
           for (int kb = 0; kb < shape.kb; ++kb, ++it) {
             const int s = it % kNS;
             const uint32_t ph = (it / kNS) & 1u;
@@ -674,16 +708,37 @@ __global__ void onehot_dw_kernel(const __nv_bfloat16* __restrict__ Hc,
 // ------------------------------------------------------------- host side
 struct Layout {
   int cap_pad, n_tiles, n_splits, chunk_rows, n_chunks, ldz;
-  size_t off_term, off_g, off_zt, off_pm, off_ps, off_mref, off_cs, off_ovf, off_hc, off_hs,
-      off_dz, total;
+  size_t off_term, off_g, off_zt, off_pm, off_ps, off_mref, off_cs, off_ovf, off_prog, off_hc,
+      off_hs, off_dz, total;
 };
+
+// Number of vocabulary splits.  Work units of equal length keep the CTAs that sweep the
+// same split in step with each other, which is what lets them share W tiles in L2 (units
+// that differ by a tile drift apart over hundreds of waves and every W tile is then
+// fetched from DRAM several times).  So prefer a divisor of the tile count that gives
+// 8..32 tiles per split, closest to kTilesPerSplit; otherwise fall back to near-equal.
+int pick_splits(int n_tiles) {
+  int best = 0, best_gap = 1 << 30;
+  for (int s = 1; s <= n_tiles; ++s) {
+    if (n_tiles % s != 0) continue;
+    const int per = n_tiles / s;
+    if (per < 8 || per > 32) continue;
+    const int gap = per > kTilesPerSplit ? per - kTilesPerSplit : kTilesPerSplit - per;
+    if (gap < best_gap) {
+      best_gap = gap;
+      best = s;
+    }
+  }
+  if (best > 0) return best;
+  return (n_tiles + kTilesPerSplit - 1) / kTilesPerSplit;
+}
 
 Layout make_layout(const nat_loss_params& p, int64_t cap) {
   Layout L;
   const int64_t c1 = cap > 0 ? cap : 1;
   L.cap_pad = (int)((c1 + kRowPad - 1) / kRowPad * kRowPad);
   L.n_tiles = (p.V + BN - 1) / BN;
-  L.n_splits = (L.n_tiles + kTilesPerSplit - 1) / kTilesPerSplit;
+  L.n_splits = pick_splits(L.n_tiles);
   L.chunk_rows = L.cap_pad < kChunkRows ? L.cap_pad : kChunkRows;
   L.n_chunks = (L.cap_pad + L.chunk_rows - 1) / L.chunk_rows;
   L.ldz = (p.V + 63) / 64 * 64;
@@ -701,6 +756,7 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   L.off_mref = take(sizeof(float) * L.cap_pad);
   L.off_cs = take(sizeof(float) * L.cap_pad);
   L.off_ovf = take(sizeof(int32_t) * L.n_chunks);
+  L.off_prog = take(sizeof(unsigned long long) * kMaxPairs);
   off = align_up(off, 1024);
   L.off_hc = take(sizeof(__nv_bfloat16) * (size_t)L.cap_pad * p.d);
   L.off_hs = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * p.d);
@@ -829,9 +885,15 @@ int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p
 template <int MODE>
 int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2,
               const TcParams& p, int m_blocks128, int per_block, cudaStream_t stream) {
+  // Every launch gets a fresh epoch, so progress marks left by earlier launches (or
+  // whatever the workspace held before) compare as "not there yet" or are overwritten
+  // by their owner's first tile; either way they cannot stall this launch for long.
+  static unsigned long long epoch_counter = 0;
+  TcParams q = p;
+  q.epoch = (++epoch_counter) & 0x7FFFFFull;
   if (pair_slots() > 0)
-    return launch_tc_impl<MODE, 2>(a, b2, p, ((m_blocks128 + 1) / 2) * per_block, stream);
-  return launch_tc_impl<MODE, 1>(a, b1, p, m_blocks128 * per_block, stream);
+    return launch_tc_impl<MODE, 2>(a, b2, q, ((m_blocks128 + 1) / 2) * per_block, stream);
+  return launch_tc_impl<MODE, 1>(a, b1, q, m_blocks128 * per_block, stream);
 }
 
 TokenCtx make_ctx(const LossArgs& a) {
@@ -853,6 +915,7 @@ struct Ws {
   WorkspaceHead* head;
   float *term, *g, *zt, *pm, *ps, *mref, *cs;
   int32_t* ovf;
+  unsigned long long* prog;
   __nv_bfloat16 *hc, *hs, *dz;
 };
 
@@ -868,6 +931,7 @@ Ws carve(void* ws, const Layout& L) {
   w.mref = reinterpret_cast<float*>(b + L.off_mref);
   w.cs = reinterpret_cast<float*>(b + L.off_cs);
   w.ovf = reinterpret_cast<int32_t*>(b + L.off_ovf);
+  w.prog = reinterpret_cast<unsigned long long*>(b + L.off_prog);
   w.hc = reinterpret_cast<__nv_bfloat16*>(b + L.off_hc);
   w.hs = reinterpret_cast<__nv_bfloat16*>(b + L.off_hs);
   w.dz = reinterpret_cast<__nv_bfloat16*>(b + L.off_dz);
@@ -903,6 +967,8 @@ TcParams base_params(const LossArgs& a, const Layout& L, const Ws& w) {
   p.flag = nullptr;
   p.run_if = 0;
   p.ovf = nullptr;
+  p.progress = w.prog;
+  p.epoch = 0;
   return p;
 }
 
