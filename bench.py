@@ -242,18 +242,31 @@ def run_ours(args, w):
         st.compact(cu)
         n_sel_total += int(st.n_sel.item())
 
+    # ---- per-kernel durations: the same K steps again with event pairs around every
+    # tensor-core launch (kept out of the timed region above)
+    from paper_2603_06619_b200 import nat as _nat
+    trace = None
+    if w.dtype == "bf16":
+        _nat.nat_trace_begin()
+        for i in range(args.steps):
+            main_step(batch, args.warmup + i)
+        trace = _nat.nat_trace_end()
+        sync_all()
+
     # ---- the other route, for the record (same batch, same offsets, 1 warm-up)
     other = step_two_pass if args.route == "single" else step
-    other(batch, 0)
-    sync_all()
-    o_begin = torch.cuda.Event(enable_timing=True)
-    o_end = torch.cuda.Event(enable_timing=True)
-    o_begin.record()
-    for i in range(args.steps):
-        other(batch, args.warmup + i)
-    o_end.record()
-    sync_all()
-    other_ms = o_begin.elapsed_time(o_end)
+    other_ms = float("nan")
+    if not args.skip_other_route:
+        other(batch, 0)
+        sync_all()
+        o_begin = torch.cuda.Event(enable_timing=True)
+        o_end = torch.cuda.Event(enable_timing=True)
+        o_begin.record()
+        for i in range(args.steps):
+            other(batch, args.warmup + i)
+        o_end.record()
+        sync_all()
+        other_ms = o_begin.elapsed_time(o_end)
 
     # ---- end to end: the step's inputs come from pinned host memory
     host = {k: batch[k].cpu().pin_memory() for k in ("hidden", "targets", "old_logp", "rewards")}
@@ -298,18 +311,45 @@ def run_ours(args, w):
     executed = counted if args.route == "single" else 8.0 * n_step * dV
     call_tflops = counted / (loss_call_ms * 1e-3) / 1e12
     step_tflops = counted / (step_ms * 1e-3) / 1e12
-    cap_pad = (n_tot + 127) // 128 * 128
+    cap_pad = (n_tot + 255) // 256 * 256
     n_chunks = (cap_pad + min(cap_pad, 8192) - 1) // min(cap_pad, 8192)
     sel_launches = 1 + (1 if w.sel_mode == "urs" else 2) + 3
     if w.dtype == "f32":
         launches = sel_launches + 2 + 3
     elif args.route == "single":
-        launches = sel_launches + 2 + 9 * n_chunks + 3
+        launches = sel_launches + 2 + 9 * n_chunks + 3      # gather, references; per chunk 9; tail 3
     else:
         launches = sel_launches + 4 + (3 + 3 * n_chunks)
     kernel = ("nat_tc_kernel<kE|kDh|kDw> (the launches inside nat_policy_loss_fwd_bwd)"
               if args.route == "single" else
               "nat_tc_kernel<kFwd|kDz|kDh|kDw> (nat_policy_loss_fwd + nat_policy_loss_bwd)")
+    roof_ms, roof_flops, per_kernel, traffic = loss_call_ms, counted, None, None
+    if trace:
+        # counted FLOPs of one step per kernel kind: the forward's 2NdV belongs to kFwd or kE,
+        # dH and dW have 2NdV each, the recompute (kDz) and the one-tile reference pass have none
+        unit = 2.0 * n_step * dV
+        credit = {"e": unit, "dh": unit, "dw": unit, "dz": 0.0,
+                  "fwd": unit if args.route == "two" else 0.0}
+        active = -(-int(n_step) // 8192)
+        per_kernel = {}
+        for kind, (ms, n_launch) in trace.items():
+            if n_launch == 0:
+                continue
+            ms_step = ms / args.steps
+            per_kernel[kind] = {
+                "ms_per_step": ms_step, "launches_per_step": n_launch / args.steps,
+                "ms_per_active_launch": ms_step / active if kind != "fwd" or args.route == "two"
+                else None,
+                "tflops_counted": credit[kind] / (ms_step * 1e-3) / 1e12 if ms_step > 0 else None}
+        top = max(per_kernel, key=lambda k: per_kernel[k]["ms_per_step"])
+        kernel = "nat_tc_kernel<%s>" % {"e": "kE", "dh": "kDh", "dw": "kDw", "dz": "kDz",
+                                         "fwd": "kFwd"}[top]
+        roof_ms, roof_flops = per_kernel[top]["ms_per_step"], credit[top]
+        # DRAM bytes per launch (one 8192-row chunk of this head) from the ncu capture
+        # summarised in profiles/nat_tc_kernel_qwen3_8b_chunk.md; null for other shapes
+        if w.name == "qwen3_8b":
+            traffic = {"e": 8.4e9, "dh": 19.3e9, "dw": 18.8e9}.get(top)
+    call_tflops = roof_flops / (roof_ms * 1e-3) / 1e12
 
     line = {
         "metric": METRIC, "value": n_all / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
@@ -330,17 +370,20 @@ def run_ours(args, w):
             "sustained": step_tflops / peak,
             "datasheet_2250": step_tflops / 2250.0},
         "loss_call_ms": loss_call_ms, "loss": loss_val, "device_status": status,
-        "other_route": {"route": "two pass" if args.route == "single" else "single pass",
-                        "ms_per_step": other_ms / args.steps,
-                        "tflops_counted": counted / (other_ms / args.steps * 1e-3) / 1e12},
+        "other_route": None if args.skip_other_route else {
+            "route": "two pass" if args.route == "single" else "single pass",
+            "ms_per_step": other_ms / args.steps,
+            "tflops_counted": counted / (other_ms / args.steps * 1e-3) / 1e12},
         "roofline": {
             "kernel": kernel, "bound": "tensor", "achieved": call_tflops, "peak": peak,
             "unit": "TFLOP/s", "frac": call_tflops / peak,
             "peak_source": f"{peak_kind} bf16_tflops_sustained (of measured)"
             if peak_kind == "measured" else "fallback (of fallback)",
-            "flops": "counted 6*N_sel*d*V per step (2 forward + 4 backward), divided by the "
-                     "event-timed duration of the loss call(s), small kernels included",
-            "traffic": None},
+            "flops": ("counted 2*N_sel*d*V per step for this kernel, divided by its event-timed "
+                      "duration summed over the step's launches (nat_trace_begin/end)") if trace
+            else "counted 6*N_sel*d*V per step divided by the event-timed loss call(s)",
+            "traffic": traffic, "traffic_unit": "DRAM bytes per launch (8192-row chunk)"},
+        "per_kernel": per_kernel,
         "e2e": {"value": n_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": 4, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": launches * args.steps,
@@ -369,6 +412,8 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-other-route", action="store_true",
+                    help="do not also time the route that was not selected")
     ap.add_argument("--route", default="single", choices=["single", "two"],
                     help="single: nat_policy_loss_fwd_bwd; two: forward then backward calls")
     args = ap.parse_args()

@@ -235,6 +235,25 @@ int nat_policy_loss_fwd_bwd(const nat_loss_params* params /* host */, const void
                             float* loss, float* logp, float* lse, void* dHidden, float* dW,
                             void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * Per-kernel timing of the bf16 loss kernels (a measurement aid of this library;
+ * the paper has no counterpart).  Between nat_trace_begin() and nat_trace_end()
+ * every tensor-core kernel launch made by the loss entry points is bracketed by
+ * a pair of CUDA events on the caller's stream.  nat_trace_end() waits for those
+ * events (it synchronises with the work traced so far), adds up the elapsed
+ * milliseconds and the launch counts per kernel kind into two HOST arrays of
+ * NAT_TRACE_KINDS entries (either may be NULL), releases the events and stops
+ * tracing.  Tracing creates CUDA events; leave it off in allocation-free code.
+ * ------------------------------------------------------------------------- */
+#define NAT_TRACE_KINDS 5
+#define NAT_TRACE_FWD 0 /* S = H W^T with online log-sum-exp (forward; also the row references) */
+#define NAT_TRACE_DZ 1  /* recomputed S -> softmax gradient (two-pass backward) */
+#define NAT_TRACE_DH 2  /* dHidden contraction */
+#define NAT_TRACE_DW 3  /* dW contraction */
+#define NAT_TRACE_E 4   /* single-pass S -> softmax numerators */
+int nat_trace_begin(void);
+int nat_trace_end(float* ms_by_kind /* host */, int32_t* launches_by_kind /* host */);
+
 #ifdef __cplusplus
 }
 #endif

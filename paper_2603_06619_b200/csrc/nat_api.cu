@@ -142,4 +142,10 @@ int nat_policy_loss_fwd_bwd(const nat_loss_params* params, const void* hidden, c
   return params->dtype == NAT_F32 ? nat::loss_f32_fwd_bwd(a) : nat::loss_bf16_fwd_bwd(a);
 }
 
+int nat_trace_begin(void) { return nat::trace_begin(); }
+
+int nat_trace_end(float* ms_by_kind, int32_t* launches_by_kind) {
+  return nat::trace_end(ms_by_kind, launches_by_kind);
+}
+
 }  // extern "C"

@@ -70,5 +70,7 @@ size_t loss_bf16_workspace_bytes(const nat_loss_params& p, int64_t cap);
 int loss_bf16_fwd(const LossArgs& a);
 int loss_bf16_bwd(const LossArgs& a);
 int loss_bf16_fwd_bwd(const LossArgs& a);
+int trace_begin();
+int trace_end(float* ms_by_kind, int32_t* launches_by_kind);
 
 }  // namespace nat

@@ -29,6 +29,9 @@
 // Every mbarrier wait is bounded; a wait that runs out raises the block's
 // abort flag and NAT_DEV_TIMEOUT in the workspace's status word.
 #include <cuda_bf16.h>
+
+#include <mutex>
+#include <vector>
 #include <cstdlib>
 
 #include "nat_tc.cuh"
@@ -848,6 +851,15 @@ int pair_slots() {
   return slots;
 }
 
+// ---- optional per-kernel timing (nat_trace_begin / nat_trace_end) ----------------
+struct TraceSpan {
+  int kind;
+  cudaEvent_t t0, t1;
+};
+std::mutex g_trace_mutex;
+bool g_trace_on = false;
+std::vector<TraceSpan> g_trace_spans;
+
 template <int MODE, int CTAS>
 int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, int max_units,
                    cudaStream_t stream) {
@@ -876,7 +888,23 @@ int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  bool traced = false;
+  TraceSpan span{MODE, nullptr, nullptr};
+  {
+    std::lock_guard<std::mutex> lock(g_trace_mutex);
+    traced = g_trace_on;
+  }
+  if (traced) {
+    NAT_CUDA(cudaEventCreate(&span.t0));
+    NAT_CUDA(cudaEventCreate(&span.t1));
+    NAT_CUDA(cudaEventRecord(span.t0, stream));
+  }
   NAT_CUDA(cudaLaunchKernelEx(&cfg, nat_tc_kernel<MODE, CTAS>, a, b, p));
+  if (traced) {
+    NAT_CUDA(cudaEventRecord(span.t1, stream));
+    std::lock_guard<std::mutex> lock(g_trace_mutex);
+    g_trace_spans.push_back(span);
+  }
   return NAT_OK;
 }
 
@@ -1145,6 +1173,44 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
     if ((s = launch_onehot(a, w)) != NAT_OK) return s;
   }
   return launch_loss_reduce(w.term, a.n_sel, a.cap, a.loss, w.head, a.stream);
+}
+
+int trace_begin() {
+  std::lock_guard<std::mutex> lock(g_trace_mutex);
+  for (TraceSpan& sp : g_trace_spans) {
+    cudaEventDestroy(sp.t0);
+    cudaEventDestroy(sp.t1);
+  }
+  g_trace_spans.clear();
+  g_trace_on = true;
+  return NAT_OK;
+}
+
+int trace_end(float* ms_by_kind, int32_t* launches_by_kind) {
+  std::vector<TraceSpan> spans;
+  {
+    std::lock_guard<std::mutex> lock(g_trace_mutex);
+    g_trace_on = false;
+    spans.swap(g_trace_spans);
+  }
+  for (int k = 0; k < NAT_TRACE_KINDS; ++k) {
+    if (ms_by_kind) ms_by_kind[k] = 0.f;
+    if (launches_by_kind) launches_by_kind[k] = 0;
+  }
+  int status = NAT_OK;
+  for (TraceSpan& sp : spans) {
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(sp.t1);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, sp.t0, sp.t1);
+    if (e != cudaSuccess) status = check_cuda(e, "nat_trace_end");
+    if (sp.kind >= 0 && sp.kind < NAT_TRACE_KINDS) {
+      if (ms_by_kind) ms_by_kind[sp.kind] += ms;
+      if (launches_by_kind) launches_by_kind[sp.kind] += 1;
+    }
+    cudaEventDestroy(sp.t0);
+    cudaEventDestroy(sp.t1);
+  }
+  return status;
 }
 
 }  // namespace nat

@@ -21,8 +21,10 @@ SYMBOLS = (
     "nat_status_string", "nat_last_error", "nat_version", "nat_grpo_adv", "nat_select",
     "nat_compact_workspace_bytes", "nat_compact", "nat_policy_loss_workspace_bytes",
     "nat_policy_loss_fwd", "nat_policy_loss_bwd", "nat_compact_static",
-    "nat_compact_static_max_tokens", "nat_policy_loss_fwd_bwd",
+    "nat_compact_static_max_tokens", "nat_policy_loss_fwd_bwd", "nat_trace_begin",
+    "nat_trace_end",
 )
+TRACE_KINDS = ("fwd", "dz", "dh", "dw", "e")
 
 
 class NatError(RuntimeError):
@@ -73,6 +75,9 @@ def load():
         [vp] * 6 + [ctypes.c_size_t, vp]
     lib.nat_policy_loss_fwd_bwd.argtypes = [ctypes.POINTER(LossParams)] + [vp] * 10 + [i64] + \
         [vp] * 7 + [ctypes.c_size_t, vp]
+    lib.nat_trace_begin.restype = ctypes.c_int
+    lib.nat_trace_end.restype = ctypes.c_int
+    lib.nat_trace_end.argtypes = [vp, vp]
     for name in ("nat_grpo_adv", "nat_select", "nat_compact", "nat_policy_loss_fwd",
                  "nat_policy_loss_bwd", "nat_policy_loss_fwd_bwd"):
         getattr(lib, name).restype = ctypes.c_int
@@ -173,6 +178,18 @@ def nat_policy_loss_fwd_bwd(params, hidden, W, targets, old_logp, adv, pi, cu_se
         _ptr(pi), _ptr(cu_seqlens), _ptr(sel_idx), _ptr(sel_resp), _ptr(n_sel), n_sel_cap,
         _ptr(dloss), _ptr(loss), _ptr(logp), _ptr(lse), _ptr(dHidden), _ptr(dW), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _stream()))
+
+
+def nat_trace_begin():
+    _check(load().nat_trace_begin())
+
+
+def nat_trace_end():
+    """Returns {kind: (milliseconds, launches)} for the tensor-core kernels traced."""
+    ms = (ctypes.c_float * len(TRACE_KINDS))()
+    cnt = (ctypes.c_int32 * len(TRACE_KINDS))()
+    _check(load().nat_trace_end(ms, cnt))
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(TRACE_KINDS)}
 
 
 def alloc_workspace(nbytes, device):

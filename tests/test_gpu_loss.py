@@ -183,3 +183,19 @@ def test_fused_accumulate_and_dloss():
     assert torch.equal(loss, st.loss)
     assert parity.rel_fro(st.dW.cpu().numpy(), -base.cpu().numpy()) < 1e-2
     assert parity.rel_fro(st.dH[:n].float().cpu().numpy(), -2 * baseH[:n].float().cpu().numpy()) < 1e-2
+
+
+def test_trace_reports_per_kernel_time():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = parity.gpu_step(w, batch, 0, 0, fused=True)
+    nat.nat_trace_begin()
+    st.loss_fwd_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"],
+                    batch["cu_seqlens"])
+    tr = nat.nat_trace_end()
+    assert tr["e"][1] == 1 and tr["e"][0] > 0 and tr["dh"][0] > 0 and tr["dw"][0] > 0
+    assert tr["dz"][1] == 1            # the predicated redo was launched (and did nothing)
+    # tracing is off again: nothing is recorded by later calls
+    st.loss_fwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], batch["cu_seqlens"])
+    nat.nat_trace_begin()
+    assert all(v == (0.0, 0) for v in nat.nat_trace_end().values())
