@@ -54,6 +54,7 @@ constexpr int kRowPad = 256;                       // compact rows are padded to
 enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3, kE = 4 };
 
 constexpr float kWindow = 60.f;  // largest S - mref the single-pass route accepts
+constexpr float kWindowSum = 1.1420073898156842e26f;  // e^60
 
 struct TcParams {
   const int32_t* n_sel;
@@ -447,20 +448,26 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
           } else if (MODE == kE) {
             const int nv = ncols - col0 < 32 ? ncols - col0 : 32;
             const float nm2 = lk * kLog2e;
-            const float live = row_ok ? 1.f : 0.f;
-            float part = 0.f, tmax = -INFINITY;
+            float part = 0.f;
             uint32_t packed[16];
+            if (row_ok) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const float t0 = fmaf(v[2 * j], kLog2e, -nm2);
-              const float t1 = fmaf(v[2 * j + 1], kLog2e, -nm2);
-              float e0 = live * fast_exp2(t0), e1 = live * fast_exp2(t1);
-              if (2 * j < nv) { part += e0; tmax = fmaxf(tmax, t0); }
-              if (2 * j + 1 < nv) { part += e1; tmax = fmaxf(tmax, t1); }
-              packed[j] = pack_bf16(e0, e1);
+              for (int j = 0; j < 16; ++j) {
+                const float e0 = fast_exp2(fmaf(v[2 * j], kLog2e, -nm2));
+                const float e1 = fast_exp2(fmaf(v[2 * j + 1], kLog2e, -nm2));
+                if (2 * j < nv) part += e0;
+                if (2 * j + 1 < nv) part += e1;
+                packed[j] = pack_bf16(e0, e1);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) packed[j] = 0u;  // rows past the last token stay zero
             }
             s_run += part;
-            if (row_ok && tmax > kWindow * kLog2e) over = true;
+            // Any numerator above 2^(kWindow log2 e) makes the chunk's sum exceed it too, so one
+            // compare per chunk catches every row that leaves the window (and at worst flags a
+            // few rows that were still inside it, which only costs the redo).
+            if (part > kWindowSum) over = true;
             if (y >= col0 && y < col0 + 32) {
 #pragma unroll
               for (int j = 0; j < 32; ++j)

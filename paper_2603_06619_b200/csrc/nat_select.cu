@@ -104,75 +104,110 @@ __global__ void cut_kernel(SelConst c, int B, const int32_t* __restrict__ cu,
   cut_len[i] = L;
 }
 
-// One thread per 16 consecutive packed tokens.
+// Owner search restricted to responses lo..hi (cu[lo] <= n < cu[hi + 1]).
+__device__ __forceinline__ int owner_between(const int32_t* __restrict__ cu, int lo, int hi,
+                                             int64_t n) {
+  ++hi;  // invariant: cu[lo] <= n < cu[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(cu + mid) <= n) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// One block per 4096 consecutive packed tokens, one thread per 16 of them (so a thread
+// reuses each Philox block for up to four tokens).  The mask leaves as one 16-byte store
+// per thread; pi is transposed through shared memory so that every warp store covers 512
+// contiguous bytes.
+constexpr int kSelBlockTokens = kSelThreads * kTokPerThread;  // 4096
+constexpr int kPiPad = kTokPerThread + 1;                     // 17: conflict-free rows
+
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
               const int32_t* __restrict__ cut_len, uint8_t* __restrict__ mask,
               float* __restrict__ pi) {
-  const int64_t n0 = ((int64_t)blockIdx.x * kSelThreads + threadIdx.x) * kTokPerThread;
-  if (n0 >= n_tot) return;
-  const int cnt = (int)min((int64_t)kTokPerThread, n_tot - n0);
-  int i = owner_of(cu, B, n0);
-  int64_t start = cu[i], end = cu[i + 1];
-  int L = 0, C = 0;
-  float den = 1.f;
-  auto enter_response = [&]() {
-    if (c.mode != NAT_SEL_URS) {
-      L = cut_len[i];
-      const int T = (int)(end - start);
-      C = (c.mode == NAT_SEL_RPC) ? min(max(c.min_cut, 1), T) : T;
-      den = (float)(T - C + 1);
-    }
-  };
-  enter_response();
-  uint32_t cached_blk = 0xFFFFFFFFu;
-  int cached_resp = -1;
-  Philox4 rnd = {0, 0, 0, 0};
-
-  alignas(16) uint8_t m[kTokPerThread];
-  alignas(16) float pr[kTokPerThread];
-#pragma unroll
-  for (int j = 0; j < kTokPerThread; ++j) {
-    m[j] = 0;
-    pr[j] = 0.f;
-    if (j < cnt) {
-      const int64_t n = n0 + j;
-      while (n >= end) {  // skips empty responses too
-        ++i;
-        start = end;
-        end = cu[i + 1];
-        if (n < end) enter_response();
-      }
-      const uint32_t t0 = (uint32_t)(n - start);  // t - 1
-      if (c.mode == NAT_SEL_URS) {
-        const uint32_t blk = t0 >> 2;
-        if (blk != cached_blk || i != cached_resp) {
-          rnd = philox4x32_10(blk, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1);
-          cached_blk = blk;
-          cached_resp = i;
-        }
-        const uint32_t lane = t0 & 3u;
-        const uint32_t x = lane == 0 ? rnd.x : lane == 1 ? rnd.y : lane == 2 ? rnd.z : rnd.w;
-        m[j] = ((uint64_t)x < c.thr) ? 1 : 0;
-        pr[j] = c.pi_urs;
-      } else {
-        const int t = (int)t0 + 1;
-        m[j] = (t <= L) ? 1 : 0;
+  __shared__ float pi_s[kSelThreads * kPiPad];
+  __shared__ int range_s[2];
+  const int64_t nb0 = (int64_t)blockIdx.x * kSelBlockTokens;
+  const int cnt_block = (int)min((int64_t)kSelBlockTokens, n_tot - nb0);
+  if (threadIdx.x == 0) {
+    range_s[0] = owner_of(cu, B, nb0);
+    range_s[1] = owner_of(cu, B, nb0 + cnt_block - 1);
+  }
+  __syncthreads();
+  const int64_t n0 = nb0 + (int64_t)threadIdx.x * kTokPerThread;
+  if (n0 < n_tot) {
+    const int cnt = (int)min((int64_t)kTokPerThread, n_tot - n0);
+    int i = owner_between(cu, range_s[0], range_s[1], n0);
+    int64_t start = cu[i], end = cu[i + 1];
+    int L = 0, C = 0;
+    float den = 1.f;
+    auto enter_response = [&]() {
+      if (c.mode != NAT_SEL_URS) {
+        L = cut_len[i];
         const int T = (int)(end - start);
-        pr[j] = (t <= C) ? 1.f : __fdiv_rn((float)(T - t + 1), den);
+        C = (c.mode == NAT_SEL_RPC) ? min(max(c.min_cut, 1), T) : T;
+        den = (float)(T - C + 1);
       }
+    };
+    enter_response();
+    uint32_t cached_blk = 0xFFFFFFFFu;
+    int cached_resp = -1;
+    Philox4 rnd = {0, 0, 0, 0};
+
+    alignas(16) uint8_t m[kTokPerThread];
+    float* pr = pi_s + threadIdx.x * kPiPad;
+#pragma unroll
+    for (int j = 0; j < kTokPerThread; ++j) {
+      m[j] = 0;
+      float pv = 0.f;
+      if (j < cnt) {
+        const int64_t n = n0 + j;
+        while (n >= end) {  // skips empty responses too
+          ++i;
+          start = end;
+          end = cu[i + 1];
+          if (n < end) enter_response();
+        }
+        const uint32_t t0 = (uint32_t)(n - start);  // t - 1
+        if (c.mode == NAT_SEL_URS) {
+          const uint32_t blk = t0 >> 2;
+          if (blk != cached_blk || i != cached_resp) {
+            rnd = philox4x32_10(blk, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1);
+            cached_blk = blk;
+            cached_resp = i;
+          }
+          const uint32_t lane = t0 & 3u;
+          const uint32_t x = lane == 0 ? rnd.x : lane == 1 ? rnd.y : lane == 2 ? rnd.z : rnd.w;
+          m[j] = ((uint64_t)x < c.thr) ? 1 : 0;
+          pv = c.pi_urs;
+        } else {
+          const int t = (int)t0 + 1;
+          m[j] = (t <= L) ? 1 : 0;
+          const int T = (int)(end - start);
+          pv = (t <= C) ? 1.f : __fdiv_rn((float)(T - t + 1), den);
+        }
+      }
+      pr[j] = pv;
+    }
+    if (cnt == kTokPerThread) {
+      *reinterpret_cast<uint4*>(mask + n0) = *reinterpret_cast<const uint4*>(m);
+    } else {
+      for (int j = 0; j < cnt; ++j) mask[n0 + j] = m[j];
     }
   }
-  if (cnt == kTokPerThread) {
-    *reinterpret_cast<uint4*>(mask + n0) = *reinterpret_cast<const uint4*>(m);
+  __syncthreads();
+  // pi: element e of the block sits at pi_s[(e / 16) * 17 + e % 16]
+  if (cnt_block == kSelBlockTokens) {
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      *reinterpret_cast<float4*>(pi + n0 + 4 * q) = *reinterpret_cast<const float4*>(pr + 4 * q);
-  } else {
-    for (int j = 0; j < cnt; ++j) {
-      mask[n0 + j] = m[j];
-      pi[n0 + j] = pr[j];
+    for (int k = 0; k < kTokPerThread / 4; ++k) {
+      const int e = (k * kSelThreads + threadIdx.x) * 4;
+      const float* src = pi_s + (e / kTokPerThread) * kPiPad + (e % kTokPerThread);
+      *reinterpret_cast<float4*>(pi + nb0 + e) = make_float4(src[0], src[1], src[2], src[3]);
     }
+  } else {
+    for (int e = threadIdx.x; e < cnt_block; e += kSelThreads)
+      pi[nb0 + e] = pi_s[(e / kTokPerThread) * kPiPad + (e % kTokPerThread)];
   }
 }
 
@@ -270,7 +305,15 @@ compact_write_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
   __shared__ int warp_tot[kCmpThreads / 32];
   __shared__ int thread_excl[kCmpThreads];
   __shared__ uint32_t thread_bits[kCmpThreads];
+  __shared__ int32_t idx_s[kChunk];
+  __shared__ int32_t resp_s[kChunk];
+  __shared__ int range_s[2];
   const int64_t chunk0 = (int64_t)blockIdx.x * kChunk;
+  if (threadIdx.x == 0) {  // responses that own the chunk's first and last token
+    const int64_t last = min(chunk0 + (int64_t)kChunk, n_tot) - 1;
+    range_s[0] = owner_of(cu, B, chunk0);
+    range_s[1] = owner_of(cu, B, last);
+  }
   const int64_t n0 = chunk0 + (int64_t)threadIdx.x * kTokPerThread;
   const uint32_t bits = (n0 < n_tot) ? load_mask_bits(mask, n0, n_tot) : 0u;
   const int c = __popc(bits);
@@ -290,19 +333,31 @@ compact_write_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
   thread_bits[threadIdx.x] = bits;
   __syncthreads();
 
+  // The chunk's selected tokens are consecutive in the output lists: stage them in
+  // shared memory, then write them out with fully coalesced stores.
   if (bits != 0u) {
-    int i = owner_of(cu, B, n0);
+    int i = owner_between(cu, range_s[0], range_s[1], n0);
     int64_t end = cu[i + 1];
-    int64_t k = excl;
+    int k = excl - base;
     for (int j = 0; j < kTokPerThread; ++j) {
       if ((bits >> j) & 1u) {
         const int64_t n = n0 + j;
         while (n >= end) end = cu[++i + 1];
-        if (k < cap) {
-          sel_idx[k] = (int32_t)n;
-          sel_resp[k] = i;
-        }
+        idx_s[k] = (int32_t)n;
+        resp_s[k] = i;
         ++k;
+      }
+    }
+  }
+  __syncthreads();
+  {
+    int total = 0;
+    for (int w = 0; w < kCmpThreads / 32; ++w) total += warp_tot[w];
+    for (int e = threadIdx.x; e < total; e += kCmpThreads) {
+      const int64_t k = (int64_t)base + e;
+      if (k < cap) {
+        sel_idx[k] = idx_s[e];
+        sel_resp[k] = resp_s[e];
       }
     }
   }
@@ -381,8 +436,7 @@ static int select_impl(const nat_select_params* sp, int32_t B, const int32_t* cu
     NAT_LAUNCH_CHECK("cut_kernel");
   }
   if (n_tot > 0) {
-    const int64_t per_block = (int64_t)kSelThreads * kTokPerThread;
-    const unsigned grid = (unsigned)((n_tot + per_block - 1) / per_block);
+    const unsigned grid = (unsigned)((n_tot + kSelBlockTokens - 1) / kSelBlockTokens);
     select_kernel<<<grid, kSelThreads, 0, stream>>>(c, B, cu_seqlens, n_tot, cut_len, mask, pi);
     NAT_LAUNCH_CHECK("select_kernel");
   }

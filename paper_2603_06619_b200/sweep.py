@@ -1,0 +1,156 @@
+"""Measurement helpers beyond the headline benchmark.
+
+    python -m paper_2603_06619_b200.sweep fraction   # time vs selected-token fraction
+    python -m paper_2603_06619_b200.sweep stress     # select / compact GB/s at 2^28 tokens
+    python -m paper_2603_06619_b200.sweep chunk      # two row chunks of the head (for ncu)
+
+`fraction` runs the single-pass loss on the Qwen3-8B-shaped batch under every
+selection setting of the sweep (URS p = 0.25 .. 1, RPC with the paper's minimum
+cut of 100, deterministic 50 % truncation) and fits time = a + b * fraction.
+`stress` times selection and compaction on a stream long enough (2^28 tokens)
+for HBM bandwidth, not launch latency, to be what is measured.  Both print
+markdown tables.
+"""
+import argparse
+import json
+import os
+import statistics
+
+import numpy as np
+import torch
+
+from . import workloads as wl
+from .step import NatStep
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+def _time(fn, reps, warmup=1):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def fraction_sweep(name="qwen3_8b", reps=2, seed=0):
+    w = wl.WORKLOADS[name]
+    batch = wl.make_batch(w, seed=seed, device="cuda")
+    n_tot = batch["n_tot"]
+    st = NatStep(w.P, w.G, w.d, w.V, torch.bfloat16, n_tot)
+    cu = batch["cu_seqlens"]
+    st.grpo_adv(batch["rewards"])
+    settings = [("URS p=0.25", dict(mode="urs", p=0.25)), ("URS p=0.5", dict(mode="urs", p=0.5)),
+                ("URS p=0.75", dict(mode="urs", p=0.75)),
+                ("full tokens (URS p=1)", dict(mode="urs", p=1.0)),
+                ("RPC C=100", dict(mode="rpc", min_cut=100)),
+                ("Det. trunc. 50%", dict(mode="det", beta=0.5))]
+    peaks, kind = _peaks()
+    rows = []
+    for label, kw in settings:
+        st.select(cu, seed=seed, **kw)
+        st.compact(cu)
+        n_sel = int(st.n_sel.item())
+        args = (batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+        ms = _time(lambda: st.loss_fwd_bwd(*args), reps)
+        assert st.status() & ~4 == 0
+        tf = 6.0 * n_sel * w.d * w.V / (ms * 1e-3) / 1e12
+        rows.append((label, n_sel, n_sel / n_tot, ms, tf))
+    x = np.array([r[2] for r in rows])
+    y = np.array([r[3] for r in rows])
+    b, a = np.polyfit(x, y, 1)
+    resid = y - (a + b * x)
+    out = [f"Workload {name}: N_tot = {n_tot}, d = {w.d}, V = {w.V}; single-pass "
+           f"nat_policy_loss_fwd_bwd, mean of {reps} calls after 1 warm-up; peaks {kind}.", "",
+           "| selection | n_sel | fraction | ms | TFLOP/s counted | of burst peak | of sustained peak |",
+           "|---|---|---|---|---|---|---|"]
+    for label, n_sel, frac, ms, tf in rows:
+        out.append(f"| {label} | {n_sel} | {frac:.3f} | {ms:.1f} | {tf:.0f} | "
+                   f"{tf / peaks['bf16_tflops']:.3f} | {tf / peaks['bf16_tflops_sustained']:.3f} |")
+    out += ["", f"Least-squares fit: time = a + b * fraction with a = {a:.1f} ms, b = {b:.1f} ms "
+            f"(a/b = {a / b:.3f}); largest residual {np.abs(resid).max():.1f} ms "
+            f"({100 * np.abs(resid / y).max():.1f} % of its point)."]
+    return "\n".join(out)
+
+
+def select_compact_stress(log2_tokens=28, T=8192, reps=5):
+    n_tot = 1 << log2_tokens
+    B = n_tot // T
+    G = 8
+    P = B // G
+    cu = torch.arange(0, n_tot + 1, T, dtype=torch.int32, device="cuda")
+    st = NatStep(P, G, 64, 512, torch.float32, n_tot, want_grads=False)
+    peaks, kind = _peaks()
+    hbm = peaks["hbm_gbs"]
+    out = [f"N_tot = 2^{log2_tokens} tokens, B = {B} responses of {T}; mean of {reps} calls; "
+           f"HBM peak {hbm:.0f} GB/s ({kind}).", "",
+           "| call | selected fraction | ms | algorithmic bytes | GB/s | of HBM peak |",
+           "|---|---|---|---|---|---|"]
+    for label, kw in (("URS p=0.5", dict(mode="urs", p=0.5)), ("RPC C=100", dict(mode="rpc", min_cut=100))):
+        ms = _time(lambda: st.select(cu, seed=1, **kw), reps)
+        nbytes = 5.0 * n_tot
+        st.compact(cu)
+        frac = int(st.n_sel.item()) / n_tot
+        out.append(f"| nat_select {label} | {frac:.3f} | {ms:.3f} | 5 B/token (mask + pi written) | "
+                   f"{nbytes / ms / 1e6:.0f} | {nbytes / ms / 1e6 / hbm:.3f} |")
+        msc = _time(lambda: st.compact(cu), reps)
+        cbytes = (1.0 + 8.0 * frac) * n_tot
+        out.append(f"| nat_compact after {label} | {frac:.3f} | {msc:.3f} | 1 B/token read + 8 B per "
+                   f"selected token written | {cbytes / msc / 1e6:.0f} | {cbytes / msc / 1e6 / hbm:.3f} |")
+    st.grpo_adv(torch.zeros(B, device="cuda"))
+    ms = _time(lambda: st.grpo_adv(torch.zeros(B, device="cuda")), reps)
+    out.append(f"| nat_grpo_adv ({P} groups of {G}) | - | {ms:.3f} | launch bound | - | - |")
+    return "\n".join(out)
+
+
+def one_chunk_sample(name="qwen3_8b", rows=16384, calls=2):
+    """The single-pass loss on `rows` tokens of the workload's head (two 8192-row chunks by
+    default): a small case for profiler captures whose launches have the benchmark's
+    per-launch shape (one chunk of this head per launch)."""
+    base = wl.WORKLOADS[name]
+    T = rows // base.G
+    w = wl.variant(base, P=1, sel_mode="urs", p=1.0, length_law="uniform", len_lo=T, len_hi=T)
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = NatStep(w.P, w.G, w.d, w.V, torch.bfloat16, batch["n_tot"])
+    cu = batch["cu_seqlens"]
+    st.grpo_adv(batch["rewards"])
+    st.select(cu, "urs", p=1.0)
+    st.compact(cu)
+    for _ in range(calls):
+        st.loss_fwd_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+        torch.cuda.synchronize()
+    assert st.status() & ~4 == 0
+    return f"{int(st.n_sel.item())} rows of the {name} head, {calls} single-pass calls"
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("what", choices=["fraction", "stress", "chunk"])
+    ap.add_argument("--workload", default="qwen3_8b")
+    ap.add_argument("--reps", type=int, default=2)
+    ap.add_argument("--log2-tokens", type=int, default=28)
+    args = ap.parse_args()
+    if args.what == "chunk":
+        print(one_chunk_sample(args.workload))
+    elif args.what == "fraction":
+        print(fraction_sweep(args.workload, reps=args.reps))
+    else:
+        print(select_compact_stress(log2_tokens=args.log2_tokens, reps=max(args.reps, 5)))
+
+
+if __name__ == "__main__":
+    main()
