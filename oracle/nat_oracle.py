@@ -194,7 +194,8 @@ def _token_weights(pi, cu_seqlens, sel_idx, sel_resp):
 
 
 def policy_loss_fwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, sel_resp,
-                    clip_lo=0.2, clip_hi=0.2, hidden_is_compact=False):
+                    clip_lo=0.2, clip_hi=0.2, hidden_is_compact=False, kl_beta=0.0,
+                    ref_logp=None):
     """Loss and per-token statistics over the selected tokens.
 
     For selected token n (row h_n of ``hidden``):
@@ -204,7 +205,10 @@ def policy_loss_fwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, 
         r      = exp(logp - old_logp[n])
         S      = min(r A, clip(r, 1-clip_lo, 1+clip_hi) A),  A = adv[resp(n)]
         w      = 1 / (pi[n] * T_resp(n) * B)
-        loss   = - sum_n w S
+        L      = S - kl_beta * (logp - ref_logp[n])     (Eq. grpo-token-loss with the
+                 per-token KL taken in the sampled-token form of its footnote;
+                 kl_beta = 0, the paper's experimental setting, drops it)
+        loss   = - sum_n w L
 
     ``hidden`` is [N_tot, d] (rows picked by sel_idx) or, with
     hidden_is_compact, [n_sel, d] with row k belonging to sel_idx[k].
@@ -229,14 +233,18 @@ def policy_loss_fwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, 
     ratio = np.exp(logp - old)
     clipped = np.minimum(np.maximum(ratio, 1.0 - clip_lo), 1.0 + clip_hi)
     S = np.minimum(ratio * A, clipped * A)
-    loss = -float(np.sum(w * S))
-    return dict(loss=loss, logp=logp, lse=lse, ratio=ratio, S=S, w=w)
+    L = S
+    if kl_beta != 0.0:
+        ref = np.asarray(ref_logp, dtype=np.float64)[sel_idx]
+        L = S - float(kl_beta) * (logp - ref)
+    loss = -float(np.sum(w * L))
+    return dict(loss=loss, logp=logp, lse=lse, ratio=ratio, S=S, w=w, L=L)
 
 
 # --------------------------------------------------------------------------
 # Policy loss over the selected tokens: backward
 # --------------------------------------------------------------------------
-def grad_coeff(ratio, A, w, clip_lo, clip_hi, dloss=1.0):
+def grad_coeff(ratio, A, w, clip_lo, clip_hi, dloss=1.0, kl_beta=0.0):
     """g_n = d loss / d logp_n.
 
     The min in the surrogate picks r*A (which has gradient A*r w.r.t. logp)
@@ -244,12 +252,13 @@ def grad_coeff(ratio, A, w, clip_lo, clip_hi, dloss=1.0):
     A < 0 and r < 1-clip_lo, where the surrogate is flat.  A = 0 gives zero.
     """
     active = ((A > 0) & (ratio <= 1.0 + clip_hi)) | ((A < 0) & (ratio >= 1.0 - clip_lo))
-    return np.where(active, -dloss * w * A * ratio, 0.0)
+    # the KL term -kl_beta (logp - ref_logp) has derivative -kl_beta w.r.t. logp
+    return np.where(active, -dloss * w * A * ratio, 0.0) + dloss * w * float(kl_beta)
 
 
 def policy_loss_bwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, sel_resp,
                     clip_lo=0.2, clip_hi=0.2, hidden_is_compact=False, dloss=1.0,
-                    want_dW=True):
+                    want_dW=True, kl_beta=0.0, ref_logp=None):
     """Gradients of ``policy_loss_fwd``'s loss.
 
         dz[n, v]  = g_n (1[v = y_n] - softmax(z_n)[v])
@@ -261,7 +270,7 @@ def policy_loss_bwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, 
     dW_dense that exclude the one-hot target terms.
     """
     fwd = policy_loss_fwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, sel_resp,
-                          clip_lo, clip_hi, hidden_is_compact)
+                          clip_lo, clip_hi, hidden_is_compact, kl_beta, ref_logp)
     W64 = np.asarray(W, dtype=np.float64)
     V, d = W64.shape
     sel_idx = np.asarray(sel_idx, dtype=np.int64)
@@ -269,7 +278,7 @@ def policy_loss_bwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, 
     n_sel = sel_idx.shape[0]
     y = np.asarray(targets, dtype=np.int64)[sel_idx]
     A = np.asarray(adv, dtype=np.float64)[sel_resp]
-    g = grad_coeff(fwd["ratio"], A, fwd["w"], clip_lo, clip_hi, dloss)
+    g = grad_coeff(fwd["ratio"], A, fwd["w"], clip_lo, clip_hi, dloss, kl_beta)
     dH = np.zeros((n_sel, d))
     dH_dense = np.zeros((n_sel, d))
     dW = np.zeros((V, d)) if want_dW else None

@@ -307,3 +307,44 @@ def test_rpc_mask_covariance():
     for s in range(T):
         for t in range(s, T):
             assert abs(cov[s, t] - p[t] * (1 - p[s])) < 1e-12
+
+
+# ---- optional KL term (Eq. grpo-token-loss, sampled-token form of its footnote) ----
+def test_kl_term_closed_form_and_gradient():
+    w, b = _tiny(old_noise=0.3, lengths=[5, 9, 4, 7, 6, 8, 3, 10], rewards=[1, 0, 0, 1, 0, 1, 0, 0])
+    mask, pi, _ = select(SEL_URS, b["cu_seqlens"], p=0.5, seed=2)
+    si, sr, so, n = compact(mask, b["cu_seqlens"])
+    rng = np.random.default_rng(3)
+    ref_logp = b["old_logp"].astype(np.float64) + rng.normal(0, 0.1, b["n_tot"])
+    beta = 0.05
+    base = _run(b, mask, pi)
+    out = _run(b, mask, pi, kl_beta=beta, ref_logp=ref_logp)
+    # loss differs from the beta = 0 loss by + beta * sum_n w_n (logp_n - ref_n)
+    want = base["loss"] + beta * np.sum(base["w"] * (base["logp"] - ref_logp[si]))
+    assert abs(out["loss"] - want) < 1e-12
+    # with ref_logp equal to the current logp the penalty vanishes but its gradient does not
+    ref_same = b["old_logp"].astype(np.float64).copy()
+    ref_same[si] = base["logp"]
+    same = _run(b, mask, pi, kl_beta=beta, ref_logp=ref_same)
+    assert abs(same["loss"] - base["loss"]) < 1e-12
+    np.testing.assert_allclose(same["g"] - base["g"], beta * base["w"], rtol=1e-12)
+
+    # finite differences of the full loss
+    def loss_at(H, W):
+        return policy_loss_fwd(H, W, b["targets"], b["old_logp"], b["adv"], pi, b["cu_seqlens"],
+                               si, sr, kl_beta=beta, ref_logp=ref_logp)["loss"]
+    H0 = b["hidden"].astype(np.float64)
+    W0 = b["W"].astype(np.float64)
+    step = 1e-6
+    for _ in range(8):
+        k, j, v = rng.integers(n), rng.integers(w.d), rng.integers(w.V)
+        Hp, Hm = H0.copy(), H0.copy()
+        Hp[si[k], j] += step
+        Hm[si[k], j] -= step
+        fd = (loss_at(Hp, W0) - loss_at(Hm, W0)) / (2 * step)
+        assert abs(fd - out["dH"][k, j]) < 1e-6 * np.abs(out["dH"]).max() + 1e-9
+        Wp, Wm = W0.copy(), W0.copy()
+        Wp[v, j] += step
+        Wm[v, j] -= step
+        fd = (loss_at(H0, Wp) - loss_at(H0, Wm)) / (2 * step)
+        assert abs(fd - out["dW"][v, j]) < 1e-6 * np.abs(out["dW"]).max() + 1e-9
