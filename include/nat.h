@@ -152,7 +152,9 @@ int nat_compact_static(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, cons
  *   z = W h (V logits, fp32 accumulation), lse = log sum_v exp z_v,
  *   logp = z[targets[n]] - lse,  r = exp(logp - old_logp[n]),
  *   S = min(r A_i, clip(r, 1-clip_lo, 1+clip_hi) A_i),
- *   w = 1 / (pi[n] T_i B),   loss = - sum_k w S.
+ *   L = S - kl_beta (logp - ref_logp[n])   (Eq. grpo-token-loss; the per-token KL in the
+ *       sampled-token form of the paper's footnote; kl_beta = 0 by default),
+ *   w = 1 / (pi[n] T_i B),   loss = - sum_k w L.
  * The logits are never written to memory.
  *
  * dtype NAT_BF16: hidden, W, dHidden are bfloat16 and the projection runs on
@@ -182,6 +184,11 @@ typedef struct {
   float clip_hi;
   int32_t hidden_is_compact;
   int32_t accumulate_dW; /* backward: 0 overwrite dW, 1 add to it */
+  float kl_beta;         /* coefficient of the KL term of Eq. grpo-token-loss; 0 (the paper's
+                            experimental setting) leaves the term out */
+  int32_t reserved;      /* set to 0 */
+  const float* ref_logp; /* device float32 [n_tot]: log-probability of each token under the
+                            reference policy; read only when kl_beta != 0 (else may be NULL) */
 } nat_loss_params;
 
 size_t nat_policy_loss_workspace_bytes(const nat_loss_params* params /* host */,
@@ -196,8 +203,8 @@ int nat_policy_loss_fwd(const nat_loss_params* params /* host */, const void* hi
 
 /* ---------------------------------------------------------------------------
  * Backward of the loss above (the gradient of Eq. ht-estimator, Appendix A).
- * With g_k = -dloss w A r 1[surrogate not saturated] (saturated: A > 0 and
- * r > 1+clip_hi, or A < 0 and r < 1-clip_lo; A = 0 gives 0):
+ * With g_k = -dloss w (A r 1[surrogate not saturated] - kl_beta) (saturated: A > 0 and
+ * r > 1+clip_hi, or A < 0 and r < 1-clip_lo; A = 0 gives 0 for the first term):
  *   dz[k, v] = g_k (1[v = y_k] - exp(z_v - lse_k))      (z recomputed)
  *   dHidden[k, :] = sum_v dz[k, v] W[v, :]     compact: row k <-> sel_idx[k]
  *   dW[v, :]      = sum_k dz[k, v] h_k          float32 [V, d]

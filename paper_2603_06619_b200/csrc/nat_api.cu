@@ -39,6 +39,8 @@ static int validate(const char* who, const nat_loss_params* p, const LossArgs& a
     return fail(NAT_ERR_UNSUPPORTED, "%s: unknown dtype %d", who, p->dtype);
   if (!(p->clip_lo >= 0.f) || !(p->clip_hi >= 0.f))
     return fail(NAT_ERR_INVALID_ARG, "%s: clip bounds must be >= 0", who);
+  if (p->kl_beta != 0.f && !p->ref_logp)
+    return fail(NAT_ERR_INVALID_ARG, "%s: kl_beta != 0 needs ref_logp", who);
   if (a.cap < 0 || a.cap > 0x7FFFFFFFll)
     return fail(NAT_ERR_INVALID_ARG, "%s: n_sel_cap out of range", who);
   if (!a.hidden || !a.W || !a.targets || !a.old_logp || !a.adv || !a.pi || !a.cu_seqlens ||

@@ -943,6 +943,8 @@ TokenCtx make_ctx(const LossArgs& a) {
   c.B = a.p.B;
   c.clip_lo = a.p.clip_lo;
   c.clip_hi = a.p.clip_hi;
+  c.kl_beta = a.p.kl_beta;
+  c.ref_logp = a.p.ref_logp;
   return c;
 }
 

@@ -24,12 +24,14 @@ struct TokenCtx {
   const int32_t* sel_resp;
   int B;
   float clip_lo, clip_hi;
+  float kl_beta;          // 0: no KL term
+  const float* ref_logp;  // read only when kl_beta != 0
 };
 
 // For selected token k with log-probability logp:
 //   r = exp(logp - old_logp), S = min(r A, clip(r) A), w = 1 / (pi T B)
-//   term = -w S               (the token's share of the loss)
-//   g    = -dloss w A r       if the surrogate is not saturated, else 0
+//   term = -w (S - kl_beta (logp - ref_logp))      (the token's share of the loss)
+//   g    = -dloss w (A r [surrogate not saturated] - kl_beta)
 __device__ __forceinline__ void token_eval(const TokenCtx& c, int k, float logp, float dloss,
                                            float* term, float* g) {
   const int n = c.sel_idx[k];
@@ -41,9 +43,15 @@ __device__ __forceinline__ void token_eval(const TokenCtx& c, int k, float logp,
   const float hi = 1.f + c.clip_hi, lo = 1.f - c.clip_lo;
   const float rc = fminf(fmaxf(r, lo), hi);
   const float S = fminf(r * A, rc * A);
-  *term = -w * S;
   const bool live = (A > 0.f && r <= hi) || (A < 0.f && r >= lo);
-  *g = live ? -dloss * w * A * r : 0.f;
+  float t = -w * S;
+  float gk = live ? -dloss * w * A * r : 0.f;
+  if (c.kl_beta != 0.f) {
+    t += w * c.kl_beta * (logp - c.ref_logp[n]);
+    gk += dloss * w * c.kl_beta;
+  }
+  *term = t;
+  *g = gk;
 }
 
 // loss = sum_k term[k] in a fixed order: each of 1024 threads adds a strided

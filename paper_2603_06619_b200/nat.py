@@ -39,7 +39,9 @@ class SelectParams(ctypes.Structure):
 class LossParams(ctypes.Structure):
     _fields_ = [("d", ctypes.c_int32), ("V", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("B", ctypes.c_int32), ("clip_lo", ctypes.c_float), ("clip_hi", ctypes.c_float),
-                ("hidden_is_compact", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32)]
+                ("hidden_is_compact", ctypes.c_int32), ("accumulate_dW", ctypes.c_int32),
+                ("kl_beta", ctypes.c_float), ("reserved", ctypes.c_int32),
+                ("ref_logp", ctypes.c_void_p)]
 
 
 _lib = None
@@ -142,10 +144,12 @@ def nat_compact_static(B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offset
 
 
 def loss_params(d, V, dtype, B, clip_lo=0.2, clip_hi=0.2, hidden_is_compact=False,
-                accumulate_dW=False):
+                accumulate_dW=False, kl_beta=0.0, ref_logp=None):
+    """ref_logp (float32 device tensor [n_tot]) must outlive the calls that use the params."""
     dtype = {torch.float32: NAT_F32, torch.bfloat16: NAT_BF16}.get(dtype, dtype)
     return LossParams(d=d, V=V, dtype=dtype, B=B, clip_lo=clip_lo, clip_hi=clip_hi,
-                      hidden_is_compact=int(hidden_is_compact), accumulate_dW=int(accumulate_dW))
+                      hidden_is_compact=int(hidden_is_compact), accumulate_dW=int(accumulate_dW),
+                      kl_beta=kl_beta, reserved=0, ref_logp=_ptr(ref_logp))
 
 
 def nat_policy_loss_workspace_bytes(params, n_sel_cap):

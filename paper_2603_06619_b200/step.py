@@ -11,7 +11,8 @@ from . import nat
 
 class NatStep:
     def __init__(self, P, G, d, V, dtype, n_tot, device="cuda", n_sel_cap=None,
-                 clip_lo=0.2, clip_hi=0.2, eps=1e-6, hidden_is_compact=False, want_grads=True):
+                 clip_lo=0.2, clip_hi=0.2, eps=1e-6, hidden_is_compact=False, want_grads=True,
+                 kl_beta=0.0, ref_logp=None):
         self.P, self.G, self.B = P, G, P * G
         self.d, self.V, self.dtype = d, V, dtype
         self.n_tot = int(n_tot)
@@ -29,7 +30,9 @@ class NatStep:
         self.sel_offsets = torch.empty(self.B + 1, dtype=i32, device=dev)
         self.n_sel = torch.zeros(1, dtype=i32, device=dev)
         self.compact_ws = nat.alloc_workspace(nat.nat_compact_workspace_bytes(self.n_tot), dev)
-        self.params = nat.loss_params(d, V, dtype, self.B, clip_lo, clip_hi, hidden_is_compact)
+        self.ref_logp = ref_logp            # keeps the tensor alive while params point at it
+        self.params = nat.loss_params(d, V, dtype, self.B, clip_lo, clip_hi, hidden_is_compact,
+                                      kl_beta=kl_beta, ref_logp=ref_logp)
         self.loss = torch.zeros(1, dtype=f32, device=dev)
         self.logp = torch.empty(max(self.cap, 1), dtype=f32, device=dev)
         self.lse = torch.empty(max(self.cap, 1), dtype=f32, device=dev)

@@ -66,21 +66,22 @@ def check_selection(st, ref, w):
 
 
 def check_loss(st, ref_sel, nb, w, backward=True, hidden_is_compact=False, clip=(0.2, 0.2),
-               hidden_np=None):
+               hidden_np=None, kl_beta=0.0, ref_logp=None):
     """Element-by-element comparison of loss, logp, lse, dHidden, dW with the oracle."""
     n = ref_sel["n_sel"]
     hidden = nb["hidden"] if hidden_np is None else hidden_np
     fn = oracle.policy_loss_bwd if backward else oracle.policy_loss_fwd
     ref = fn(hidden, nb["W"], nb["targets"], nb["old_logp"], ref_sel["adv"], ref_sel["pi"],
              nb["cu_seqlens"], ref_sel["sel_idx"], ref_sel["sel_resp"], clip_lo=clip[0],
-             clip_hi=clip[1], hidden_is_compact=hidden_is_compact)
+             clip_hi=clip[1], hidden_is_compact=hidden_is_compact, kl_beta=kl_beta,
+             ref_logp=ref_logp)
     assert st.status() & ~4 == 0      # the informational fallback bit may be set
     got_logp = st.logp[:n].cpu().numpy()
     got_lse = st.lse[:n].cpu().numpy()
     assert np.abs(got_logp - ref["logp"]).max(initial=0) <= TOL_LOGP
     assert np.abs(got_lse - ref["lse"]).max(initial=0) <= TOL_LOGP
     loss = float(st.loss.item())
-    floor = 1e-2 * float(np.sum(ref["w"] * np.abs(ref["S"])))
+    floor = 1e-2 * float(np.sum(ref["w"] * np.abs(ref["L"])))
     assert abs(loss - ref["loss"]) <= TOL_LOSS * max(abs(ref["loss"]), floor), (loss, ref["loss"])
     out = dict(loss=loss, ref_loss=ref["loss"])
     if backward:

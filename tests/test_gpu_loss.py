@@ -199,3 +199,26 @@ def test_trace_reports_per_kernel_time():
     st.loss_fwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], batch["cu_seqlens"])
     nat.nat_trace_begin()
     assert all(v == (0.0, 0) for v in nat.nat_trace_end().values())
+
+
+@pytest.mark.parametrize("name,fused", [("tiny", False), ("mid", False), ("mid", True)])
+def test_kl_term(name, fused):
+    # Eq. grpo-token-loss with kl_beta > 0 (sampled-token KL against a reference policy)
+    w = wl.variant(wl.WORKLOADS[name], old_noise=0.3)
+    batch = wl.make_batch(w, seed=5, device="cuda")
+    g = torch.Generator(device="cuda")
+    g.manual_seed(11)
+    ref_logp = batch["old_logp"] + 0.1 * torch.randn(batch["n_tot"], generator=g, device="cuda")
+    nb = wl.to_numpy(batch)
+    ref_sel = parity.oracle_selection(w, nb, 5, 0)
+    st = parity.gpu_step(w, batch, 5, 0, fused=fused, kl_beta=0.05, ref_logp=ref_logp)
+    parity.check_selection(st, ref_sel, w)
+    out, ref = parity.check_loss(st, ref_sel, nb, w, kl_beta=0.05,
+                                 ref_logp=ref_logp.cpu().numpy())
+    base = oracle.policy_loss_fwd(nb["hidden"], nb["W"], nb["targets"], nb["old_logp"],
+                                  ref_sel["adv"], ref_sel["pi"], nb["cu_seqlens"],
+                                  ref_sel["sel_idx"], ref_sel["sel_resp"])
+    assert abs(ref["loss"] - base["loss"]) > 1e-4          # the term is not a no-op here
+    # kl_beta != 0 without a reference is refused
+    with pytest.raises(nat.NatError):
+        parity.gpu_step(w, batch, 5, 0, fused=fused, kl_beta=0.05, ref_logp=None)
