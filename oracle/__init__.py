@@ -14,6 +14,10 @@ Parity status of each function (what pins it to something other than itself):
   select            pinned: the paper's closed forms for the survival
                     probabilities, E[L], exact enumeration of every cut value
                     in rational arithmetic, binomial frequency test for URS.
+  select_survival   pinned: boundary values of the 24-bit draw against the exact count
+                    ceil(p 2^24), the uniform-cutoff schedule reproducing the uniform law,
+                    prefix structure, and exhaustive enumeration of a geometric cut law
+                    showing the HT estimator unbiased (Proposition 1).
   compact           pinned: brute-force list comprehension, segment structure
                     for prefix modes.
   policy_loss_fwd   pinned: softmax rows sum to one, scipy log_softmax,
@@ -31,6 +35,7 @@ from .nat_oracle import (  # noqa: F401
     SEL_DET,
     grpo_adv,
     select,
+    select_survival,
     compact,
     policy_loss_fwd,
     policy_loss_bwd,

@@ -142,6 +142,40 @@ def select(mode, cu_seqlens, *, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
     return mask, pi, cut_len
 
 
+def select_survival(cu_seqlens, surv, *, seed=0, offset=0):
+    """Random Prefix Cutting under a caller-given survival schedule (Eq. rpc-mask,
+    Eq. rpc-survival with a general cut law q_i).
+
+    ``surv[n]`` is p_{i,t} = Pr(L_i >= t) for packed token n: non-increasing inside a
+    response, 1 at its first token, positive at its last.  Response i draws one uniform
+    u = (x0 >> 8) * 2^-24 from the Philox block with counter (0, i, 2, offset_lo); then
+    L_i >= t  <=>  u < p_{i,t}, so m_t = [u < surv[n]] (a prefix because surv is monotone)
+    and Pr(L_i >= t) = ceil(p_{i,t} 2^24) / 2^24, within 2^-24 of the schedule.
+    The inclusion probabilities are the schedule itself.
+
+    Returns (mask uint8 [N_tot], cut_len int32 [B]).
+    """
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    surv = np.asarray(surv, dtype=np.float32)
+    B = cu.shape[0] - 1
+    mask = np.zeros(int(cu[B]), dtype=np.uint8)
+    cut_len = np.zeros(B, dtype=np.int32)
+    k0, k1, off_lo = _key(seed, offset)
+    for i in range(B):
+        lo, hi = int(cu[i]), int(cu[i + 1])
+        if hi == lo:
+            continue
+        p = surv[lo:hi]
+        if p[0] != 1.0 or np.any(np.diff(p) > 0) or p[-1] <= 0:
+            raise ValueError("survival schedule must start at 1, not increase and stay positive")
+        x0, _, _, _ = philox4x32_10(0, i, 2, off_lo, k0, k1)
+        u = np.float32(int(x0) >> 8) * np.float32(2.0 ** -24)
+        m = u < p
+        mask[lo:hi] = m.astype(np.uint8)
+        cut_len[i] = int(m.sum())
+    return mask, cut_len
+
+
 # --------------------------------------------------------------------------
 # Compaction of the selected token indices
 # --------------------------------------------------------------------------

@@ -348,3 +348,32 @@ def test_kl_term_closed_form_and_gradient():
         Wm[v, j] -= step
         fd = (loss_at(H0, Wp) - loss_at(H0, Wm)) / (2 * step)
         assert abs(fd - out["dW"][v, j]) < 1e-6 * np.abs(out["dW"]).max() + 1e-9
+
+
+def test_general_cut_law_enumeration_is_unbiased():
+    """Eq. rpc-survival with a non-uniform q: cuts weighted q(l) = p_l - p_{l+1} give the
+    full-token loss and gradient in expectation when pi = p (Proposition 1)."""
+    w, b = _tiny(old_noise=0.3, lengths=[6, 9, 5, 7, 4, 8, 3, 10], rewards=[1, 0, 0, 1, 0, 1, 0, 0])
+    cu = b["cu_seqlens"]
+    surv = np.concatenate([np.maximum(0.8 ** np.arange(T), 0.1) for T in np.diff(cu)])
+    surv[cu[:-1]] = 1.0
+    pi = surv.astype(np.float32)
+    for i in range(w.B):
+        T = cu[i + 1] - cu[i]
+        p = pi[cu[i]:cu[i + 1]].astype(np.float64)
+        q = p - np.append(p[1:], 0.0)                 # Pr(L = l), l = 1..T
+        assert abs(q.sum() - 1.0) < 1e-12 and np.all(q >= 0)
+        only = np.zeros(b["n_tot"], dtype=np.uint8)
+        only[cu[i]:cu[i + 1]] = 1
+        full = _run(b, only, np.ones_like(pi))
+        e_loss, e_dW = 0.0, 0.0
+        for L in range(1, T + 1):
+            if q[L - 1] == 0:
+                continue
+            m = np.zeros(b["n_tot"], dtype=np.uint8)
+            m[cu[i]:cu[i] + L] = 1
+            out = _run(b, m, pi)
+            e_loss += q[L - 1] * out["loss"]
+            e_dW = e_dW + q[L - 1] * out["dW"]
+        assert abs(e_loss - full["loss"]) < 2e-7 * abs(full["loss"]) + 1e-9
+        np.testing.assert_allclose(e_dW, full["dW"], atol=2e-7 * np.abs(full["dW"]).max())

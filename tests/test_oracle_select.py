@@ -253,3 +253,60 @@ def test_compact_brute_force_and_segments():
     want = np.concatenate([np.arange(cu[i], cu[i] + cut[i]) for i in range(len(T))])
     assert np.array_equal(si, want)
     assert n == cut.sum()
+
+
+# ------------------------------------------------- general survival schedules
+from oracle import select_survival  # noqa: E402
+
+
+def _geometric_schedule(T, rho, floor):
+    p = np.maximum(rho ** np.arange(T), floor).astype(np.float32)
+    p[0] = 1.0
+    return p
+
+
+def test_survival_selection_is_a_prefix_with_the_scheduled_law():
+    rng = np.random.default_rng(7)
+    T = np.array([1, 5, 64, 300, 0, 17])
+    cu = _cu(T)
+    surv = np.concatenate([_geometric_schedule(t, 0.97, 0.05) for t in T if t > 0])
+    mask, cut = select_survival(cu, surv, seed=3, offset=1)
+    for i, Ti in enumerate(T):
+        m = mask[cu[i]:cu[i + 1]]
+        assert m.sum() == cut[i] and np.all(m[:cut[i]] == 1) and np.all(m[cut[i]:] == 0)
+        assert (cut[i] >= 1) == (Ti > 0)
+    # frequencies over many responses: Pr(L >= t) = surv_t (binomial z-test, fixed seeds)
+    Tn, R = 40, 4000
+    p = _geometric_schedule(Tn, 0.9, 0.02)
+    cuR = _cu([Tn] * R)
+    maskR, cutR = select_survival(cuR, np.tile(p, R), seed=11)
+    freq = maskR.reshape(R, Tn).mean(0)
+    z = (freq - p) / np.sqrt(np.maximum(p * (1 - p), 1e-12) / R)
+    assert np.abs(z[1:]).max() < 4.5 and freq[0] == 1.0
+    # the uniform-cutoff schedule (T-t+1)/T gives a uniform cut: E[L] = (T+1)/2
+    pu = ((Tn - np.arange(Tn)) / Tn).astype(np.float32)
+    _, cutU = select_survival(cuR, np.tile(pu, R), seed=12)
+    assert abs(cutU.mean() - (Tn + 1) / 2) < 4 * math.sqrt((Tn ** 2 - 1) / 12 / R)
+    with pytest.raises(ValueError):
+        select_survival(_cu([3]), np.array([1.0, 0.5, 0.7], dtype=np.float32))
+
+
+def test_survival_draw_boundaries_are_exact():
+    """u = k 2^-24 is kept iff k < ceil(p 2^24): checked at the two draws around the
+    boundary, found by scanning seeds for responses whose draw lands there."""
+    p_t = np.float32(0.3)
+    bound = math.ceil(float(p_t) * 2 ** 24)          # number of 24-bit draws with u < p
+    assert abs(bound / 2 ** 24 - float(p_t)) < 2 ** -24
+    surv = np.array([1.0, p_t], dtype=np.float32)
+    from oracle.philox import philox4x32_10 as ph
+    seen = {True: 0, False: 0}
+    for seed in range(400):
+        x0 = int(ph(0, 0, 2, 0, seed, 0)[0])
+        k = x0 >> 8
+        mask, cut = select_survival(_cu([2]), surv, seed=seed)
+        assert (cut[0] == 2) == (k < bound)
+        seen[k < bound] += 1
+    assert seen[True] > 50 and seen[False] > 150
+    # the comparison itself at the boundary, in float32 as the kernels do it
+    assert np.float32(bound - 1) * np.float32(2.0 ** -24) < p_t
+    assert not (np.float32(bound) * np.float32(2.0 ** -24) < p_t)
