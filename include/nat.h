@@ -99,6 +99,23 @@ int nat_select(const nat_select_params* params /* host */, int32_t B, const int3
                int64_t n_tot, uint8_t* mask, float* pi, int32_t* cut_len, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * Random Prefix Cutting under a caller-given survival schedule (Section 4:
+ * Eq. rpc-mask and Eq. rpc-survival for a general cut law q_i; Appendix B.3
+ * discusses schedules other than the uniform one).
+ *   surv float32 [n_tot]: p_{i,t} = Pr(L_i >= t) for every packed token; inside a
+ *   response it must start at 1, never increase and stay positive (not checked).
+ * Response i draws u = (x0 >> 8) 2^-24 from the Philox block with counter
+ * (0, i, 2, offset_lo), key as in nat_select; m_t = [u < surv], a prefix of
+ * length L_i because surv is monotone, and Pr(L_i >= t) = ceil(surv 2^24) / 2^24.
+ * Outputs: mask uint8 [n_tot], cut_len int32 [B] (L_i; 0 for an empty response).
+ * The inclusion probabilities are the schedule: pass `surv` as `pi` to the loss.
+ * surv and mask must be 16-byte aligned.
+ * ------------------------------------------------------------------------- */
+int nat_select_survival(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const float* surv,
+                        uint64_t seed, uint64_t offset, uint8_t* mask, int32_t* cut_len,
+                        void* stream);
+
+/* ---------------------------------------------------------------------------
  * Compaction of the selected tokens ("only included tokens contribute to
  * backpropagation", Section 1; Eq. ht-estimator sums over m = 1 only).
  *   sel_idx  int32 [cap]   ascending packed indices n with mask[n] != 0

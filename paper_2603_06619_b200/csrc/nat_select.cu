@@ -211,6 +211,61 @@ select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
   }
 }
 
+// Random prefix cutting under a caller-given survival schedule: response i draws one
+// uniform u = (x0 >> 8) 2^-24 (Philox counter (0, i, 2, offset_lo)); token t is kept iff
+// u < surv.  One thread per 16 consecutive tokens, 16-byte loads and stores; the thread
+// that sees the last kept token of a response writes its cut length.
+__global__ void __launch_bounds__(kSelThreads)
+select_survival_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
+                       const float* __restrict__ surv, uint8_t* __restrict__ mask,
+                       int32_t* __restrict__ cut_len) {
+  const int64_t n0 = ((int64_t)blockIdx.x * kSelThreads + threadIdx.x) * kTokPerThread;
+  if (n0 >= n_tot) return;
+  const int cnt = (int)min((int64_t)kTokPerThread, n_tot - n0);
+  int i = owner_of(cu, B, n0);
+  int64_t start = cu[i], end = cu[i + 1];
+  auto draw = [&]() {
+    const Philox4 r = philox4x32_10(0u, (uint32_t)i, 2u, c.off_lo, c.k0, c.k1);
+    return __fmul_rn((float)(r.x >> 8), 5.9604644775390625e-08f);  // 2^-24, exact
+  };
+  float u = draw();
+  alignas(16) float p[kTokPerThread];
+  if (cnt == kTokPerThread) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      *reinterpret_cast<float4*>(p + 4 * q) = __ldg(reinterpret_cast<const float4*>(surv + n0) + q);
+  } else {
+    for (int j = 0; j < kTokPerThread; ++j) p[j] = j < cnt ? surv[n0 + j] : 0.f;
+  }
+  alignas(16) uint8_t m[kTokPerThread];
+#pragma unroll
+  for (int j = 0; j < kTokPerThread; ++j) {
+    m[j] = 0;
+    if (j < cnt) {
+      const int64_t n = n0 + j;
+      while (n >= end) {
+        ++i;
+        start = end;
+        end = cu[i + 1];
+        if (n < end) u = draw();
+      }
+      const bool keep = u < p[j];
+      m[j] = keep ? 1 : 0;
+      if (keep) {
+        // last kept token of the response: the next one is past the end or not kept
+        const bool last = (n + 1 == end) ||
+                          !(u < (j + 1 < cnt ? p[j + 1] : __ldg(surv + n + 1)));
+        if (last) cut_len[i] = (int32_t)(n - start) + 1;
+      }
+    }
+  }
+  if (cnt == kTokPerThread) {
+    *reinterpret_cast<uint4*>(mask + n0) = *reinterpret_cast<const uint4*>(m);
+  } else {
+    for (int j = 0; j < cnt; ++j) mask[n0 + j] = m[j];
+  }
+}
+
 // ------------------------------------------------------------- compaction
 // Pass 1: selected count of each 4096-token chunk.  Pass 2: one block scans
 // the chunk counts.  Pass 3: each chunk scans its own mask and writes the
@@ -461,6 +516,34 @@ int nat_grpo_adv(int32_t P, int32_t G, const float* rewards, float eps, float* a
 int nat_select(const nat_select_params* params, int32_t B, const int32_t* cu_seqlens,
                int64_t n_tot, uint8_t* mask, float* pi, int32_t* cut_len, void* stream) {
   return nat::select_impl(params, B, cu_seqlens, n_tot, mask, pi, cut_len, (cudaStream_t)stream);
+}
+
+int nat_select_survival(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const float* surv,
+                        uint64_t seed, uint64_t offset, uint8_t* mask, int32_t* cut_len,
+                        void* stream_) {
+  using namespace nat;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (B < 0 || n_tot < 0) return fail(NAT_ERR_INVALID_ARG, "nat_select_survival: negative size");
+  if (n_tot > 0x7FFFFFFFll)
+    return fail(NAT_ERR_UNSUPPORTED, "nat_select_survival: n_tot exceeds int32");
+  if (!cu_seqlens || (B > 0 && !cut_len) || (n_tot > 0 && (!surv || !mask)))
+    return fail(NAT_ERR_INVALID_ARG, "nat_select_survival: null pointer");
+  if (((uintptr_t)surv & 15u) || ((uintptr_t)mask & 15u))
+    return fail(NAT_ERR_INVALID_ARG, "nat_select_survival: surv and mask must be 16-byte aligned");
+  if (B == 0) return NAT_OK;
+  SelConst c{};
+  c.k0 = (uint32_t)(seed & 0xFFFFFFFFull);
+  c.k1 = (uint32_t)((seed >> 32) ^ (offset >> 32));
+  c.off_lo = (uint32_t)(offset & 0xFFFFFFFFull);
+  NAT_CUDA(cudaMemsetAsync(cut_len, 0, sizeof(int32_t) * (size_t)B, stream));
+  if (n_tot > 0) {
+    const int64_t per_block = (int64_t)kSelThreads * kTokPerThread;
+    const unsigned grid = (unsigned)((n_tot + per_block - 1) / per_block);
+    select_survival_kernel<<<grid, kSelThreads, 0, stream>>>(c, B, cu_seqlens, n_tot, surv, mask,
+                                                             cut_len);
+    NAT_LAUNCH_CHECK("select_survival_kernel");
+  }
+  return NAT_OK;
 }
 
 size_t nat_compact_workspace_bytes(int64_t n_tot) {

@@ -22,7 +22,7 @@ SYMBOLS = (
     "nat_compact_workspace_bytes", "nat_compact", "nat_policy_loss_workspace_bytes",
     "nat_policy_loss_fwd", "nat_policy_loss_bwd", "nat_compact_static",
     "nat_compact_static_max_tokens", "nat_policy_loss_fwd_bwd", "nat_trace_begin",
-    "nat_trace_end",
+    "nat_trace_end", "nat_select_survival",
 )
 TRACE_KINDS = ("fwd", "dz", "dh", "dw", "e")
 
@@ -63,6 +63,9 @@ def load():
     lib.nat_version.restype = ctypes.c_int
     lib.nat_grpo_adv.argtypes = [i32, i32, vp, f32, vp, vp]
     lib.nat_select.argtypes = [ctypes.POINTER(SelectParams), i32, vp, i64, vp, vp, vp, vp]
+    lib.nat_select_survival.argtypes = [i32, vp, i64, vp, ctypes.c_uint64, ctypes.c_uint64, vp, vp,
+                                        vp]
+    lib.nat_select_survival.restype = ctypes.c_int
     lib.nat_compact_workspace_bytes.restype = ctypes.c_size_t
     lib.nat_compact_workspace_bytes.argtypes = [i64]
     lib.nat_compact.argtypes = [i32, vp, i64, vp, vp, vp, vp, vp, i64, vp, ctypes.c_size_t, vp]
@@ -118,6 +121,11 @@ def select_params(mode, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
 def nat_select(params, B, cu_seqlens, n_tot, mask, pi, cut_len):
     _check(load().nat_select(ctypes.byref(params), B, _ptr(cu_seqlens), n_tot, _ptr(mask),
                              _ptr(pi), _ptr(cut_len), _stream()))
+
+
+def nat_select_survival(B, cu_seqlens, n_tot, surv, seed, offset, mask, cut_len):
+    _check(load().nat_select_survival(B, _ptr(cu_seqlens), n_tot, _ptr(surv), seed, offset,
+                                      _ptr(mask), _ptr(cut_len), _stream()))
 
 
 def nat_compact_workspace_bytes(n_tot):

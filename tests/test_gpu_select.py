@@ -97,3 +97,57 @@ def test_invalid_arguments_are_rejected():
             nat.nat_select(nat.select_params(**kw), 2, cu, 0, buf, pi, cu)
     with pytest.raises(nat.NatError):
         nat.nat_grpo_adv(2, 0, pi, 1e-6, pi)
+
+
+# --------------------------------------------- general survival schedules (RPC)
+def _schedule(T, rho, floor):
+    p = np.maximum(rho ** np.arange(T), floor).astype(np.float32)
+    if T:
+        p[0] = 1.0
+    return p
+
+
+@pytest.mark.parametrize("lengths", [[1, 5, 64, 300, 0, 17, 4096, 33], [0, 0, 7, 0],
+                                     "qwen3_0p6b"])
+def test_survival_schedule_selection(lengths):
+    if isinstance(lengths, str):
+        lengths = wl.make_lengths(wl.WORKLOADS[lengths], 0)
+    T = np.asarray(lengths, dtype=np.int32)
+    cu = wl.cu_from_lengths(T)
+    n_tot, B = int(cu[-1]), len(T)
+    surv = np.concatenate([_schedule(int(t), 0.999 if t > 200 else 0.9, 0.03) for t in T])
+    mask = torch.full((max(n_tot, 16),), 7, dtype=torch.uint8, device="cuda")
+    cut = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    surv_d = torch.from_numpy(surv).cuda() if n_tot else torch.zeros(16, device="cuda")
+    for seed, offset in ((3, 0), (3, (5 << 32) + 9)):
+        nat.nat_select_survival(B, torch.from_numpy(cu).cuda(), n_tot, surv_d, seed, offset,
+                                mask, cut)
+        torch.cuda.synchronize()
+        ref_mask, ref_cut = oracle.select_survival(cu, surv, seed=seed, offset=offset)
+        assert np.array_equal(mask[:n_tot].cpu().numpy(), ref_mask)
+        assert np.array_equal(cut.cpu().numpy(), ref_cut)
+
+
+def test_survival_schedule_feeds_the_loss():
+    # pi = the schedule: selection, compaction and the loss agree with the oracle
+    import parity
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=2, device="cuda")
+    nb = wl.to_numpy(batch)
+    cu = nb["cu_seqlens"]
+    surv = np.concatenate([_schedule(int(t), 0.97, 0.05) for t in np.diff(cu)])
+    st = NatStep(w.P, w.G, w.d, w.V, torch.bfloat16, batch["n_tot"])
+    st.grpo_adv(batch["rewards"])
+    st.pi.copy_(torch.from_numpy(surv).cuda())
+    nat.nat_select_survival(w.B, batch["cu_seqlens"], batch["n_tot"], st.pi, 4, 0, st.mask,
+                            st.cut_len)
+    st.compact(batch["cu_seqlens"])
+    st.loss_fwd_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"],
+                    batch["cu_seqlens"])
+    torch.cuda.synchronize()
+    mask, cut = oracle.select_survival(cu, surv, seed=4)
+    si, sr, so, n = oracle.compact(mask, cu)
+    ref_sel = dict(adv=oracle.grpo_adv(nb["rewards"], w.P, w.G, 1e-6), mask=mask, pi=surv, cut=cut,
+                   sel_idx=si, sel_resp=sr, sel_offsets=so, n_sel=n)
+    parity.check_selection(st, ref_sel, w)
+    parity.check_loss(st, ref_sel, nb, w)
