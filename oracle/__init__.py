@@ -20,6 +20,8 @@ Parity status of each function (what pins it to something other than itself):
                     showing the HT estimator unbiased (Proposition 1).
   compact           pinned: brute-force list comprehension, segment structure
                     for prefix modes.
+  gather/scatter    pinned: numpy fancy indexing, scatter(gather(x)) = mask * x, and the
+                    packed prefixes being the per-response slices [cu_i, cu_i + L_i).
   policy_loss_fwd   pinned: softmax rows sum to one, scipy log_softmax,
                     old_logp == logp closed form, p = 1 full-token GRPO written
                     as an independent double loop, exhaustive enumeration of
@@ -37,6 +39,8 @@ from .nat_oracle import (  # noqa: F401
     select,
     select_survival,
     compact,
+    gather_rows,
+    scatter_rows,
     policy_loss_fwd,
     policy_loss_bwd,
 )

@@ -204,6 +204,29 @@ def compact(mask, cu_seqlens):
 
 
 # --------------------------------------------------------------------------
+# Packing for prefix-truncated computation (Section 4, "Compute savings": under
+# RPC the model only processes the prefix 1..L_i of each response)
+# --------------------------------------------------------------------------
+def gather_rows(src, sel_idx):
+    """Compact copy: row k of the result is row sel_idx[k] of ``src``."""
+    src = np.asarray(src)
+    out = np.zeros((len(sel_idx),) + src.shape[1:], dtype=src.dtype)
+    for k, n in enumerate(sel_idx):
+        out[k] = src[int(n)]
+    return out
+
+
+def scatter_rows(src, sel_idx, n_tot):
+    """Inverse placement: row sel_idx[k] of the result is row k of ``src``; every other
+    row is zero (a token that was not selected receives no gradient)."""
+    src = np.asarray(src)
+    out = np.zeros((int(n_tot),) + src.shape[1:], dtype=src.dtype)
+    for k, n in enumerate(sel_idx):
+        out[int(n)] = src[k]
+    return out
+
+
+# --------------------------------------------------------------------------
 # Policy loss over the selected tokens: forward
 #   ratio Eq. ratio, surrogate Eq. grpo-surrogate, aggregation Eq. grpo-obj,
 #   Horvitz-Thompson weights Eq. ht-estimator / Eq. rpc-ht

@@ -310,3 +310,22 @@ def test_survival_draw_boundaries_are_exact():
     # the comparison itself at the boundary, in float32 as the kernels do it
     assert np.float32(bound - 1) * np.float32(2.0 ** -24) < p_t
     assert not (np.float32(bound) * np.float32(2.0 ** -24) < p_t)
+
+
+# ------------------------------------------------------- packing of the prefixes
+def test_gather_scatter_rows():
+    from oracle import gather_rows, scatter_rows
+    rng = np.random.default_rng(4)
+    T = rng.integers(1, 40, size=9)
+    cu = _cu(T)
+    x = rng.normal(size=(cu[-1], 6)).astype(np.float32)
+    mask, _, cut = select(SEL_RPC, cu, min_cut=2, seed=8)
+    si, sr, so, n = compact(mask, cu)
+    g = gather_rows(x, si)
+    assert np.array_equal(g, x[si])                                   # library indexing
+    # under RPC the packed rows are the prefixes, and sel_offsets are their cu_seqlens
+    for i in range(len(T)):
+        assert np.array_equal(g[so[i]:so[i + 1]], x[cu[i]:cu[i] + cut[i]])
+    s = scatter_rows(g, si, cu[-1])
+    assert np.array_equal(s, x * mask[:, None])
+    assert scatter_rows(g[:0], si[:0], 5).shape == (5, 6)
