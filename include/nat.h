@@ -132,6 +132,23 @@ int nat_compact(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8
                 int64_t cap, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * Packing for prefix-truncated computation (Section 4, "Compute savings: prefix
+ * structure enables true forward truncation": under RPC the model only has to
+ * process the prefix 1..L_i of each response).
+ *   nat_gather_rows   dst[k, :] = src[sel_idx[k], :]  for k < min(*n_sel, cap)
+ *   nat_scatter_rows  dst = 0 over [n_tot, row_bytes], then
+ *                     dst[sel_idx[k], :] = src[k, :]   (e.g. compact dHidden back
+ *                     to the packed stream; unselected tokens get zero gradient)
+ * Rows are row_bytes bytes (a positive multiple of 16) of any element type;
+ * src and dst are 16-byte aligned and must not overlap.  After nat_compact under
+ * RPC or truncation, sel_offsets is the cu_seqlens of the packed prefixes.
+ * ------------------------------------------------------------------------- */
+int nat_gather_rows(const void* src, int64_t row_bytes, const int32_t* sel_idx,
+                    const int32_t* n_sel, int64_t cap, void* dst, void* stream);
+int nat_scatter_rows(const void* src, int64_t row_bytes, const int32_t* sel_idx,
+                     const int32_t* n_sel, int64_t cap, int64_t n_tot, void* dst, void* stream);
+
+/* ---------------------------------------------------------------------------
  * nat_compact_static: nat_compact without a workspace argument.  (An addition
  * of this library; the paper has no counterpart.)
  *

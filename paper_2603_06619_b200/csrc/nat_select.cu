@@ -266,6 +266,27 @@ select_survival_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_
   }
 }
 
+// ------------------------------------------------ packing selected rows
+// dst[k, :] = src[sel_idx[k], :] (gather) or dst[sel_idx[k], :] = src[k, :] (scatter) for
+// k < n_sel; rows are row_vec 16-byte vectors.  One warp per row keeps each row's
+// traffic in whole 512-byte warp transactions; the kernels are bound by HBM bandwidth
+// (row_bytes read + row_bytes written per selected row).
+__global__ void __launch_bounds__(256)
+move_rows_kernel(const uint4* __restrict__ src, int64_t row_vec,
+                 const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ n_sel,
+                 int64_t cap, int scatter, uint4* __restrict__ dst) {
+  const int64_t n = min((int64_t)*n_sel, cap);
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t k = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); k < n;
+       k += warps) {
+    const int64_t row = sel_idx[k];
+    const uint4* s = src + (scatter ? k : row) * row_vec;
+    uint4* d = dst + (scatter ? row : k) * row_vec;
+    for (int64_t j = lane; j < row_vec; j += 32) d[j] = __ldg(s + j);
+  }
+}
+
 // ------------------------------------------------------------- compaction
 // Pass 1: selected count of each 4096-token chunk.  Pass 2: one block scans
 // the chunk counts.  Pass 3: each chunk scans its own mask and writes the
@@ -544,6 +565,45 @@ int nat_select_survival(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, con
     NAT_LAUNCH_CHECK("select_survival_kernel");
   }
   return NAT_OK;
+}
+
+static int move_rows(const char* who, const void* src, int64_t row_bytes, const int32_t* sel_idx,
+                     const int32_t* n_sel, int64_t cap, int scatter, void* dst,
+                     cudaStream_t stream) {
+  using namespace nat;
+  if (row_bytes <= 0 || (row_bytes & 15) != 0)
+    return fail(NAT_ERR_INVALID_ARG, "%s: row_bytes must be a positive multiple of 16", who);
+  if (cap < 0) return fail(NAT_ERR_INVALID_ARG, "%s: negative capacity", who);
+  if (!n_sel || (cap > 0 && (!src || !dst || !sel_idx)))
+    return fail(NAT_ERR_INVALID_ARG, "%s: null pointer", who);
+  if (((uintptr_t)src & 15u) || ((uintptr_t)dst & 15u))
+    return fail(NAT_ERR_INVALID_ARG, "%s: src and dst must be 16-byte aligned", who);
+  if (cap == 0) return NAT_OK;
+  const int64_t blocks = (cap + 7) / 8;
+  const unsigned grid = (unsigned)(blocks < 148 * 8 ? blocks : 148 * 8);
+  move_rows_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint4*>(src), row_bytes / 16,
+                                             sel_idx, n_sel, cap, scatter,
+                                             reinterpret_cast<uint4*>(dst));
+  NAT_LAUNCH_CHECK("move_rows_kernel");
+  return NAT_OK;
+}
+
+int nat_gather_rows(const void* src, int64_t row_bytes, const int32_t* sel_idx,
+                    const int32_t* n_sel, int64_t cap, void* dst, void* stream) {
+  return move_rows("nat_gather_rows", src, row_bytes, sel_idx, n_sel, cap, 0, dst,
+                   (cudaStream_t)stream);
+}
+
+int nat_scatter_rows(const void* src, int64_t row_bytes, const int32_t* sel_idx,
+                     const int32_t* n_sel, int64_t cap, int64_t n_tot, void* dst, void* stream) {
+  if (n_tot < 0) return nat::fail(NAT_ERR_INVALID_ARG, "nat_scatter_rows: negative n_tot");
+  if (n_tot > 0 && row_bytes > 0 && dst) {
+    int s = nat::check_cuda(cudaMemsetAsync(dst, 0, (size_t)n_tot * (size_t)row_bytes,
+                                            (cudaStream_t)stream), "cudaMemsetAsync");
+    if (s != NAT_OK) return s;
+  }
+  return move_rows("nat_scatter_rows", src, row_bytes, sel_idx, n_sel, cap, 1, dst,
+                   (cudaStream_t)stream);
 }
 
 size_t nat_compact_workspace_bytes(int64_t n_tot) {

@@ -22,7 +22,7 @@ SYMBOLS = (
     "nat_compact_workspace_bytes", "nat_compact", "nat_policy_loss_workspace_bytes",
     "nat_policy_loss_fwd", "nat_policy_loss_bwd", "nat_compact_static",
     "nat_compact_static_max_tokens", "nat_policy_loss_fwd_bwd", "nat_trace_begin",
-    "nat_trace_end", "nat_select_survival",
+    "nat_trace_end", "nat_select_survival", "nat_gather_rows", "nat_scatter_rows",
 )
 TRACE_KINDS = ("fwd", "dz", "dh", "dw", "e")
 
@@ -66,6 +66,10 @@ def load():
     lib.nat_select_survival.argtypes = [i32, vp, i64, vp, ctypes.c_uint64, ctypes.c_uint64, vp, vp,
                                         vp]
     lib.nat_select_survival.restype = ctypes.c_int
+    lib.nat_gather_rows.argtypes = [vp, i64, vp, vp, i64, vp, vp]
+    lib.nat_gather_rows.restype = ctypes.c_int
+    lib.nat_scatter_rows.argtypes = [vp, i64, vp, vp, i64, i64, vp, vp]
+    lib.nat_scatter_rows.restype = ctypes.c_int
     lib.nat_compact_workspace_bytes.restype = ctypes.c_size_t
     lib.nat_compact_workspace_bytes.argtypes = [i64]
     lib.nat_compact.argtypes = [i32, vp, i64, vp, vp, vp, vp, vp, i64, vp, ctypes.c_size_t, vp]
@@ -126,6 +130,20 @@ def nat_select(params, B, cu_seqlens, n_tot, mask, pi, cut_len):
 def nat_select_survival(B, cu_seqlens, n_tot, surv, seed, offset, mask, cut_len):
     _check(load().nat_select_survival(B, _ptr(cu_seqlens), n_tot, _ptr(surv), seed, offset,
                                       _ptr(mask), _ptr(cut_len), _stream()))
+
+
+def _row_bytes(t):
+    return t.stride(0) * t.element_size() if t.dim() > 1 else t.element_size()
+
+
+def nat_gather_rows(src, sel_idx, n_sel, cap, dst):
+    _check(load().nat_gather_rows(_ptr(src), _row_bytes(src), _ptr(sel_idx), _ptr(n_sel), cap,
+                                  _ptr(dst), _stream()))
+
+
+def nat_scatter_rows(src, sel_idx, n_sel, cap, n_tot, dst):
+    _check(load().nat_scatter_rows(_ptr(src), _row_bytes(src), _ptr(sel_idx), _ptr(n_sel), cap,
+                                   n_tot, _ptr(dst), _stream()))
 
 
 def nat_compact_workspace_bytes(n_tot):

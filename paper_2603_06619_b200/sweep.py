@@ -114,6 +114,29 @@ def select_compact_stress(log2_tokens=28, T=8192, reps=5):
     st.grpo_adv(torch.zeros(B, device="cuda"))
     ms = _time(lambda: st.grpo_adv(torch.zeros(B, device="cuda")), reps)
     out.append(f"| nat_grpo_adv ({P} groups of {G}) | - | {ms:.3f} | launch bound | - | - |")
+    del st
+    # packing of the selected rows: the Qwen3-8B-shaped batch's hidden states under RPC
+    from . import nat
+    w = wl.WORKLOADS["qwen3_8b"]
+    T = wl.make_lengths(w, 0)
+    cu2 = torch.from_numpy(wl.cu_from_lengths(T)).cuda()
+    n2 = int(T.sum())
+    st2 = NatStep(w.P, w.G, 64, 512, torch.float32, n2, want_grads=False)
+    st2.select(cu2, "rpc", min_cut=100, seed=0)
+    st2.compact(cu2)
+    n_sel = int(st2.n_sel.item())
+    x = torch.randn(n2, w.d, device="cuda").to(torch.bfloat16)
+    packed = torch.empty_like(x)
+    full = torch.empty_like(x)
+    row = w.d * 2
+    ms = _time(lambda: nat.nat_gather_rows(x, st2.sel_idx, st2.n_sel, n2, packed), reps)
+    gb = 2.0 * n_sel * row
+    out.append(f"| nat_gather_rows ({n_sel} of {n2} rows of {row} B) | {n_sel / n2:.3f} | {ms:.3f} | "
+               f"row read + row written | {gb / ms / 1e6:.0f} | {gb / ms / 1e6 / hbm:.3f} |")
+    ms = _time(lambda: nat.nat_scatter_rows(packed, st2.sel_idx, st2.n_sel, n2, n2, full), reps)
+    sb = 2.0 * n_sel * row + 1.0 * n2 * row
+    out.append(f"| nat_scatter_rows (same, into {n2} zeroed rows) | {n_sel / n2:.3f} | {ms:.3f} | "
+               f"row read + row written + zero fill | {sb / ms / 1e6:.0f} | {sb / ms / 1e6 / hbm:.3f} |")
     return "\n".join(out)
 
 

@@ -151,3 +151,38 @@ def test_survival_schedule_feeds_the_loss():
                    sel_idx=si, sel_resp=sr, sel_offsets=so, n_sel=n)
     parity.check_selection(st, ref_sel, w)
     parity.check_loss(st, ref_sel, nb, w)
+
+
+# ----------------------------------------------------- packing of selected rows
+@pytest.mark.parametrize("d,dtype", [(64, torch.float32), (1024, torch.bfloat16), (8, torch.bfloat16)])
+def test_gather_and_scatter_rows(d, dtype):
+    w = wl.WORKLOADS["mid"]
+    T = wl.make_lengths(w, 1)
+    cu = wl.cu_from_lengths(T)
+    n_tot = int(cu[-1])
+    st = NatStep(w.P, w.G, 64, 512, torch.float32, n_tot, want_grads=False)
+    cu_d = torch.from_numpy(cu).cuda()
+    st.select(cu_d, "rpc", min_cut=3, seed=2)
+    st.compact(cu_d)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(0)
+    x = torch.randn(n_tot, d, generator=g, device="cuda").to(dtype)
+    n = int(st.n_sel.item())
+    packed = torch.full((n_tot, d), 9.0, device="cuda").to(dtype)
+    nat.nat_gather_rows(x, st.sel_idx, st.n_sel, n_tot, packed)
+    back = torch.full((n_tot, d), 9.0, device="cuda").to(dtype)
+    nat.nat_scatter_rows(packed, st.sel_idx, st.n_sel, n_tot, n_tot, back)
+    torch.cuda.synchronize()
+    si = st.sel_idx[:n].cpu().numpy()
+    xn = x.float().cpu().numpy()
+    assert np.array_equal(packed[:n].float().cpu().numpy(), oracle.gather_rows(xn, si))
+    assert torch.all(packed[n:] == 9.0)                      # rows past n_sel untouched
+    assert np.array_equal(back.float().cpu().numpy(),
+                          oracle.scatter_rows(oracle.gather_rows(xn, si), si, n_tot))
+    # the packed rows are the per-response prefixes, delimited by sel_offsets
+    so = st.sel_offsets.cpu().numpy()
+    cut = st.cut_len[:w.B].cpu().numpy()
+    assert np.array_equal(np.diff(so), cut)
+    # row_bytes must be a multiple of 16
+    assert nat.load().nat_gather_rows(x.data_ptr(), 24, st.sel_idx.data_ptr(), st.n_sel.data_ptr(), 3,
+                                      packed.data_ptr(), None) == -1
