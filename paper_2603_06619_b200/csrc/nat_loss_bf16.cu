@@ -53,7 +53,7 @@ constexpr int kRowPad = 256;                       // compact rows are padded to
 
 enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3, kE = 4 };
 
-constexpr float kWindow = 60.f;  // largest S - mref the single-pass route accepts
+// The single-pass route accepts S - mref up to 60 (numerators and their sums stay finite):
 constexpr float kWindowSum = 1.1420073898156842e26f;  // e^60
 
 struct TcParams {
@@ -102,9 +102,9 @@ struct Shape {
   int nblocks;  // N blocks (kDh, kDw) or vocabulary tiles (kFwd, kDz)
 };
 
-template <int MODE, int CTAS>
+template <int MODE, int CTAS, int SUBS>
 __device__ __forceinline__ Shape make_shape(const TcParams& p) {
-  constexpr int BMU = BM * CTAS;  // rows of the accumulator's M dimension per work unit
+  constexpr int BMU = BM * CTAS * SUBS;  // rows of the M dimension per work unit
   Shape s;
   int n = *p.n_sel;
   n = n < p.cap ? n : p.cap;
@@ -170,28 +170,35 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 constexpr float kLog2e = 1.4426950408889634f;
 
-// Shared-memory ring: CTAS = 1: 4 stages of (A 128x64 + B 256x64) = 48 KB;
+// Shared-memory ring (192 KB): CTAS = 1: stages of (A 128x64 + B 256x64) = 48 KB;
 // CTAS = 2: each CTA of the pair holds its 128 rows of A and its 128-row half
 // of B, 32 KB per stage, 6 stages.
-template <int CTAS>
+// SUBS = 2: each CTA holds two 128-row sub-tiles of A per stage (one B tile serves both,
+// which cuts the operand bytes per FLOP by a quarter) and both accumulators belong to the
+// same output tile.
+template <int CTAS, int SUBS>
 struct Ring {
   static constexpr int kBRows = BN / CTAS;
   static constexpr int kBBytes = kBRows * BK * 2;
-  static constexpr int kStage = kABytes + kBBytes;
-  static constexpr int kNum = CTAS == 1 ? 4 : 6;
+  static constexpr int kABytesS = kABytes * SUBS;
+  static constexpr int kStage = kABytesS + kBBytes;
+  static constexpr int kNum = (192 * 1024) / kStage;
   static constexpr size_t kSmem = (size_t)kNum * kStage + 1024 /*alignment*/ + 256 /*barriers*/;
 };
 
-template <int MODE, int CTAS>
+template <int MODE, int CTAS, int SUBS>
 __global__ void __launch_bounds__(kThreads, 1)
 nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
               const TcParams p) {
-  using R = Ring<CTAS>;
+  static_assert(SUBS == 1 || MODE == kDh || MODE == kDw,
+                "row state that lives across vocabulary tiles needs one sub-tile per thread");
+  using R = Ring<CTAS, SUBS>;
   constexpr int kNS = R::kNum;
-  constexpr int BMU = BM * CTAS;
+  constexpr int BMU = BM * CTAS * SUBS;
+  constexpr uint32_t kNAcc = 2 / SUBS;  // accumulator buffers: two tiles in flight, or one
   constexpr bool kAmn = (MODE == kDw);
   constexpr bool kBmn = (MODE == kDh || MODE == kDw);
-  constexpr uint32_t kIdesc = tc::instr_desc_bf16(BMU, BN, kAmn ? 1 : 0, kBmn ? 1 : 0);
+  constexpr uint32_t kIdesc = tc::instr_desc_bf16(BM * CTAS, BN, kAmn ? 1 : 0, kBmn ? 1 : 0);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -239,7 +246,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
   tc::fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  const Shape shape = make_shape<MODE, CTAS>(p);
+  const Shape shape = make_shape<MODE, CTAS, SUBS>(p);
 
   if (warp == 0) {
     // ------------------------------------------------ TMA producer
@@ -285,7 +292,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             const uint32_t ph = (it / kNS) & 1u;
             if (!tc::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
             uint8_t* a_dst = smem + (size_t)s * R::kStage;
-            uint8_t* b_dst = a_dst + kABytes;
+            uint8_t* b_dst = a_dst + R::kABytesS;
             // CTAS = 2: both CTAs' loads count on the even CTA's barrier, which its
             // own producer arms with the bytes of the whole pair.
             const uint32_t bar = CTAS == 2 ? tc::map_to_cta(tc::smem_u32(&full_bar[s]), 0)
@@ -295,19 +302,21 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
               if (CTAS == 2) tc::tma_load_2d_pair(dst, map, bar, x, y);
               else tc::tma_load_2d(dst, map, &full_bar[s], x, y);
             };
-            const int m0 = w.mb * BMU + rank * BM;            // this CTA's rows of A / D
+            const int m0 = w.mb * BMU + rank * (BM * SUBS);   // this CTA's rows of A / D
             const int n0 = nt * BN + rank * R::kBRows;        // this CTA's rows of B
             if (MODE == kFwd || MODE == kDz || MODE == kE) {
               load(a_dst, &mapA, kb * BK, p.row0 + m0);
               load(b_dst, &mapB, kb * BK, n0);
             } else if (MODE == kDh) {
-              load(a_dst, &mapA, kb * BK, m0);
+#pragma unroll
+              for (int sub = 0; sub < SUBS; ++sub)
+                load(a_dst + sub * kABytes, &mapA, kb * BK, m0 + sub * BM);
 #pragma unroll
               for (int j = 0; j < R::kBRows / 64; ++j)
                 load(b_dst + j * kBoxBytes, &mapB, n0 + j * 64, kb * BK);
             } else {
 #pragma unroll
-              for (int j = 0; j < BM / 64; ++j)
+              for (int j = 0; j < (BM * SUBS) / 64; ++j)
                 load(a_dst + j * kBoxBytes, &mapA, m0 + j * 64, kb * BK);
 #pragma unroll
               for (int j = 0; j < R::kBRows / 64; ++j)
@@ -342,33 +351,39 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
         const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
         for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt, ++tcount) {
-          const uint32_t acc = tcount & 1u;
-          const uint32_t aph = (tcount >> 1) & 1u;
+          const uint32_t acc = tcount % kNAcc;
+          const uint32_t aph = (tcount / kNAcc) & 1u;
           if (!tc::mbar_wait(&tempty_bar[acc], aph ^ 1u, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
-          const uint32_t d_tmem = tmem_base + acc * BN;
+          const uint32_t d_tmem = tmem_base + acc * SUBS * BN;
           for (int kb = 0; kb < shape.kb; ++kb, ++it) {
             const int s = it % kNS;
             const uint32_t ph = (it / kNS) & 1u;
             if (!tc::mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
             tc::fence_after_sync();
             const uint32_t a_base = tc::smem_u32(smem + (size_t)s * R::kStage);
-            const uint32_t b_base = a_base + kABytes;
+            const uint32_t b_base = a_base + R::kABytesS;
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk) {
+#pragma unroll
+              for (int sub = 0; sub < SUBS; ++sub) {
+              const uint32_t a_sub = a_base + sub * kABytes;
               // K-major: 16 elements of K are 32 bytes inside the swizzled
               // 128-byte row; 8-row groups are 1024 bytes apart.
               // MN-major: 16 rows of K are two 8-row groups 1024 bytes apart
               // (stride offset); 64-element groups along M/N are whole boxes
               // apart (leading offset).
               const uint64_t adesc =
-                  kAmn ? tc::smem_desc_sw128(a_base + kk * 2048, kBoxBytes, 1024)
-                       : tc::smem_desc_sw128(a_base + kk * 32, 16, 1024);
+                  kAmn ? tc::smem_desc_sw128(a_sub + kk * 2048, kBoxBytes, 1024)
+                       : tc::smem_desc_sw128(a_sub + kk * 32, 16, 1024);
               const uint64_t bdesc =
                   kBmn ? tc::smem_desc_sw128(b_base + kk * 2048, kBoxBytes, 1024)
                        : tc::smem_desc_sw128(b_base + kk * 32, 16, 1024);
-              if (CTAS == 2) tc::umma_bf16_pair(d_tmem, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
-              else tc::umma_bf16(d_tmem, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+              if (CTAS == 2)
+                tc::umma_bf16_pair(d_tmem + sub * BN, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+              else
+                tc::umma_bf16(d_tmem + sub * BN, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+              }
             }
             if (CTAS == 2) tc::umma_commit_pair(&empty_bar[s], 3);
             else tc::umma_commit(&empty_bar[s]);
@@ -389,36 +404,48 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     bool ok = true;
     for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
       const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
-      const int lrow = w.mb * BMU + rank * BM + q * 32 + lane;  // row inside this launch's M range
+      int lrow = 0;  // row inside this launch's M range
       // per-unit row state
       float m_run = -INFINITY, s_run = 0.f, zt_val = 0.f;
       bool zt_found = false;
       int y = -1;
       float gk = 0.f, lk = 0.f, scale = 1.f;
       bool row_ok = false, over = false;
-      if (MODE != kDw) {
-        const int k = p.row0 + lrow;
-        row_ok = k < n_valid;
-        if (row_ok) {
-          if (MODE == kFwd || MODE == kDh || MODE == kE) y = p.targets[p.sel_idx[k]];
-          if (MODE == kDz || MODE == kDh) gk = p.g[k];
-          if (MODE == kDz) lk = p.lse[k];
-          if (MODE == kE) lk = p.mref[k];
-          if (MODE == kDh && p.row_scale != nullptr) scale = p.row_scale[k];
+      auto load_row = [&](int sub) {  // this thread's row of sub-tile `sub` and its scalars
+        lrow = w.mb * BMU + rank * (BM * SUBS) + sub * BM + q * 32 + lane;
+        y = -1;
+        gk = 0.f;
+        lk = 0.f;
+        scale = 1.f;
+        if (MODE != kDw) {
+          const int k = p.row0 + lrow;
+          row_ok = k < n_valid;
+          if (row_ok) {
+            if (MODE == kFwd || MODE == kDh || MODE == kE) y = p.targets[p.sel_idx[k]];
+            if (MODE == kDz || MODE == kDh) gk = p.g[k];
+            if (MODE == kDz) lk = p.lse[k];
+            if (MODE == kE) lk = p.mref[k];
+            if (MODE == kDh && p.row_scale != nullptr) scale = p.row_scale[k];
+          }
+        } else {
+          row_ok = lrow < p.V;
         }
-      } else {
-        row_ok = lrow < p.V;
-      }
+      };
+      if (SUBS == 1) load_row(0);
       for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt, ++tcount) {
-        const uint32_t acc = tcount & 1u;
-        const uint32_t aph = (tcount >> 1) & 1u;
+        const uint32_t acc = tcount % kNAcc;
+        const uint32_t aph = (tcount / kNAcc) & 1u;
         // every lane waits (each needs the accumulator's writes visible), then the
         // warp agrees on the outcome so the aligned tensor-memory loads stay converged
         ok = __all_sync(0xFFFFFFFFu, tc::mbar_wait(&tfull_bar[acc], aph, abort_flag) ? 1 : 0) != 0;
         if (!ok) break;
         tc::fence_after_sync();
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
         const int ncols = (MODE == kFwd || MODE == kDz || MODE == kE) ? p.V : p.d;
+#pragma unroll 1
+        for (int sub = 0; sub < SUBS; ++sub) {
+        if (SUBS > 1) load_row(sub);
+        const uint32_t taddr =
+            tmem_base + ((uint32_t)(q * 32) << 16) + (acc * SUBS + (uint32_t)sub) * BN;
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           const int col0 = nt * BN + c * 32;
@@ -464,7 +491,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
               for (int j = 0; j < 16; ++j) packed[j] = 0u;  // rows past the last token stay zero
             }
             s_run += part;
-            // Any numerator above 2^(kWindow log2 e) makes the chunk's sum exceed it too, so one
+            // Any numerator above e^60 makes the chunk's sum exceed it too, so one
             // compare per chunk catches every row that leaves the window (and at worst flags a
             // few rows that were still inside it, which only costs the redo).
             if (part > kWindowSum) over = true;
@@ -531,6 +558,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             }
           }
         }
+        }  // sub
         tc::fence_before_sync();
         __syncwarp();
         if (lane == 0) {
@@ -835,12 +863,12 @@ int pair_slots() {
     slots = 0;
     int sms = 0;
     if (sm_count(&sms) == NAT_OK &&
-        cudaFuncSetAttribute(nat_tc_kernel<kFwd, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)Ring<2>::kSmem) == cudaSuccess) {
+        cudaFuncSetAttribute(nat_tc_kernel<kFwd, 2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)Ring<2, 1>::kSmem) == cudaSuccess) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)sms, 1, 1);
       cfg.blockDim = dim3(kThreads, 1, 1);
-      cfg.dynamicSmemBytes = Ring<2>::kSmem;
+      cfg.dynamicSmemBytes = Ring<2, 1>::kSmem;
       cudaLaunchAttribute attr[1];
       attr[0].id = cudaLaunchAttributeClusterDimension;
       attr[0].val.clusterDim.x = 2;
@@ -849,7 +877,7 @@ int pair_slots() {
       cfg.attrs = attr;
       cfg.numAttrs = 1;
       int clusters = 0;
-      if (cudaOccupancyMaxActiveClusters(&clusters, nat_tc_kernel<kFwd, 2>, &cfg) == cudaSuccess &&
+      if (cudaOccupancyMaxActiveClusters(&clusters, nat_tc_kernel<kFwd, 2, 1>, &cfg) == cudaSuccess &&
           clusters * 2 * 10 >= sms * 9)
         slots = clusters;
     }
@@ -867,14 +895,14 @@ std::mutex g_trace_mutex;
 bool g_trace_on = false;
 std::vector<TraceSpan> g_trace_spans;
 
-template <int MODE, int CTAS>
+template <int MODE, int CTAS, int SUBS>
 int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, int max_units,
                    cudaStream_t stream) {
   static bool configured = false;
   if (!configured) {
-    NAT_CUDA(cudaFuncSetAttribute(nat_tc_kernel<MODE, CTAS>,
+    NAT_CUDA(cudaFuncSetAttribute(nat_tc_kernel<MODE, CTAS, SUBS>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)Ring<CTAS>::kSmem));
+                                  (int)Ring<CTAS, SUBS>::kSmem));
     configured = true;
   }
   int sms = 0;
@@ -886,7 +914,7 @@ int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(groups * CTAS), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = Ring<CTAS>::kSmem;
+  cfg.dynamicSmemBytes = Ring<CTAS, SUBS>::kSmem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -906,7 +934,7 @@ int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p
     NAT_CUDA(cudaEventCreate(&span.t1));
     NAT_CUDA(cudaEventRecord(span.t0, stream));
   }
-  NAT_CUDA(cudaLaunchKernelEx(&cfg, nat_tc_kernel<MODE, CTAS>, a, b, p));
+  NAT_CUDA(cudaLaunchKernelEx(&cfg, nat_tc_kernel<MODE, CTAS, SUBS>, a, b, p));
   if (traced) {
     NAT_CUDA(cudaEventRecord(span.t1, stream));
     std::lock_guard<std::mutex> lock(g_trace_mutex);
@@ -926,9 +954,14 @@ int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2
   static unsigned long long epoch_counter = 0;
   TcParams q = p;
   q.epoch = (++epoch_counter) & 0x7FFFFFull;
+  // The long-K contractions (dH, dW) take two A sub-tiles per CTA; the vocabulary sweeps
+  // keep one, because their epilogue state lives across tiles and overlaps the next MMA.
+  constexpr int kSubs = (MODE == kDh || MODE == kDw) ? 2 : 1;
   if (pair_slots() > 0)
-    return launch_tc_impl<MODE, 2>(a, b2, q, ((m_blocks128 + 1) / 2) * per_block, stream);
-  return launch_tc_impl<MODE, 1>(a, b1, q, m_blocks128 * per_block, stream);
+    return launch_tc_impl<MODE, 2, kSubs>(a, b2, q,
+                                          ((m_blocks128 + 2 * kSubs - 1) / (2 * kSubs)) * per_block,
+                                          stream);
+  return launch_tc_impl<MODE, 1, 1>(a, b1, q, m_blocks128 * per_block, stream);
 }
 
 TokenCtx make_ctx(const LossArgs& a) {
