@@ -348,7 +348,7 @@ def run_ours(args, w):
         # DRAM bytes per launch (one 8192-row chunk of this head) from the ncu capture
         # summarised in profiles/nat_tc_kernel_qwen3_8b_chunk.md; null for other shapes
         if w.name == "qwen3_8b":
-            traffic = {"e": 8.67e9, "dh": 25.27e9, "dw": 21.44e9}.get(top)
+            traffic = {"e": 9.13e9, "dh": 10.83e9, "dw": 20.0e9}.get(top)
     call_tflops = roof_flops / (roof_ms * 1e-3) / 1e12
 
     line = {

@@ -9,7 +9,7 @@
 //   kDz   S = Hc W^T  recomputed         epilogue: -g exp(S - lse) -> bf16 into
 //                                        the bounded scratch dZ[chunk, V].
 //   kDh   dH = dZ W   (rows x d, K = V)  epilogue: + g W[y] (one-hot term) -> bf16.
-//   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 read-modify-write.
+//   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 reduction into dW (red.global.add).
 //   kE    S = Hc W^T  single-pass variant  epilogue: E = exp(S - mref) -> bf16 into the
 //                                        same scratch, row sums of E, target pick.
 //
@@ -30,6 +30,7 @@
 // abort flag and NAT_DEV_TIMEOUT in the workspace's status word.
 #include <cuda_bf16.h>
 
+#include <atomic>
 #include <mutex>
 #include <vector>
 #include <cstdlib>
@@ -545,16 +546,14 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             }
           } else {
             if (row_ok) {
-              float4* dst = reinterpret_cast<float4*>(p.dW + (size_t)lrow * p.d + col0);
+              // dW += tile: 16-byte reductions performed by the L2 (nothing comes back to
+              // the SM, so the epilogue does not wait on DRAM).  Every element is touched by
+              // one thread per launch and launches are stream-ordered: the sum's order is fixed.
+              float* dst = p.dW + (size_t)lrow * p.d + col0;
 #pragma unroll
-              for (int g4 = 0; g4 < 8; ++g4) {
-                float4 o = dst[g4];
-                o.x += v[4 * g4];
-                o.y += v[4 * g4 + 1];
-                o.z += v[4 * g4 + 2];
-                o.w += v[4 * g4 + 3];
-                dst[g4] = o;
-              }
+              for (int g4 = 0; g4 < 8; ++g4)
+                tc::red_add_f32x4(dst + 4 * g4, v[4 * g4], v[4 * g4 + 1], v[4 * g4 + 2],
+                                  v[4 * g4 + 3]);
             }
           }
         }
@@ -842,14 +841,28 @@ int make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows,
   return NAT_OK;
 }
 
+// Per-device facts are cached per device index: one process may drive several GPUs.
+constexpr int kMaxDevices = 64;
+
+int current_device(int* dev) {
+  NAT_CUDA(cudaGetDevice(dev));
+  if (*dev < 0 || *dev >= kMaxDevices)
+    return fail(NAT_ERR_UNSUPPORTED, "device index %d is beyond the %d this library tracks", *dev,
+                kMaxDevices);
+  return NAT_OK;
+}
+
 int sm_count(int* out) {
-  static int cached = 0;
-  if (!cached) {
-    int dev = 0;
-    NAT_CUDA(cudaGetDevice(&dev));
-    NAT_CUDA(cudaDeviceGetAttribute(&cached, cudaDevAttrMultiProcessorCount, dev));
+  static std::atomic<int> cached[kMaxDevices];
+  int dev = 0;
+  int s = current_device(&dev);
+  if (s != NAT_OK) return s;
+  int v = cached[dev].load();
+  if (v == 0) {
+    NAT_CUDA(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev));
+    cached[dev].store(v);
   }
-  *out = cached;
+  *out = v;
   return NAT_OK;
 }
 
@@ -858,9 +871,12 @@ int sm_count(int* out) {
 // the device can co-schedule 2-CTA clusters of this kernel on (nearly) all of its SMs;
 // otherwise (e.g. a partitioned GPU) the single-CTA kernels run.
 int pair_slots() {
-  static int slots = -1;
-  if (slots < 0) {
-    slots = 0;
+  static std::atomic<int> cached[kMaxDevices];  // 0 = unknown, -1 = none, else the count
+  int dev = 0;
+  if (current_device(&dev) != NAT_OK) return 0;
+  int slots = cached[dev].load();
+  if (slots == 0) {
+    slots = -1;
     int sms = 0;
     if (sm_count(&sms) == NAT_OK &&
         cudaFuncSetAttribute(nat_tc_kernel<kFwd, 2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -882,8 +898,9 @@ int pair_slots() {
         slots = clusters;
     }
     (void)cudaGetLastError();
+    cached[dev].store(slots);
   }
-  return slots;
+  return slots > 0 ? slots : 0;
 }
 
 // ---- optional per-kernel timing (nat_trace_begin / nat_trace_end) ----------------
@@ -898,12 +915,15 @@ std::vector<TraceSpan> g_trace_spans;
 template <int MODE, int CTAS, int SUBS>
 int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, int max_units,
                    cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
+  static std::atomic<bool> configured[kMaxDevices];
+  int dev = 0;
+  int sd = current_device(&dev);
+  if (sd != NAT_OK) return sd;
+  if (!configured[dev].load()) {
     NAT_CUDA(cudaFuncSetAttribute(nat_tc_kernel<MODE, CTAS, SUBS>,
                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)Ring<CTAS, SUBS>::kSmem));
-    configured = true;
+    configured[dev].store(true);
   }
   int sms = 0;
   int s = sm_count(&sms);
@@ -951,9 +971,9 @@ int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2
   // Every launch gets a fresh epoch, so progress marks left by earlier launches (or
   // whatever the workspace held before) compare as "not there yet" or are overwritten
   // by their owner's first tile; either way they cannot stall this launch for long.
-  static unsigned long long epoch_counter = 0;
+  static std::atomic<unsigned long long> epoch_counter{0};
   TcParams q = p;
-  q.epoch = (++epoch_counter) & 0x7FFFFFull;
+  q.epoch = (epoch_counter.fetch_add(1) + 1) & 0x7FFFFFull;
   // The long-K contractions (dH, dW) take two A sub-tiles per CTA; the vocabulary sweeps
   // keep one, because their epilogue state lives across tiles and overlaps the next MMA.
   constexpr int kSubs = (MODE == kDh || MODE == kDw) ? 2 : 1;
