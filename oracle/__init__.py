@@ -25,7 +25,7 @@ Parity status of each function (what pins it to something other than itself):
   policy_loss_fwd   pinned: softmax rows sum to one, scipy log_softmax,
                     old_logp == logp closed form, p = 1 full-token GRPO written
                     as an independent double loop, exhaustive enumeration of
-                    masks / cuts (Proposition 1).
+                    masks / cuts (Proposition 1); the optional KL term by its closed form.
   policy_loss_bwd   pinned: central finite differences of policy_loss_fwd,
                     zero column sums, exhaustive enumeration of the gradient's
                     expectation, saturated-clip zero gradient.
