@@ -3,13 +3,17 @@
     python -m paper_2603_06619_b200.sweep fraction   # time vs selected-token fraction
     python -m paper_2603_06619_b200.sweep stress     # select / compact GB/s at 2^28 tokens
     python -m paper_2603_06619_b200.sweep chunk      # two row chunks of the head (for ncu)
+    python -m paper_2603_06619_b200.sweep ceiling    # loss kernels vs library GEMMs, same operands
 
 `fraction` runs the single-pass loss on the Qwen3-8B-shaped batch under every
 selection setting of the sweep (URS p = 0.25 .. 1, RPC with the paper's minimum
 cut of 100, deterministic 50 % truncation) and fits time = a + b * fraction.
 `stress` times selection and compaction on a stream long enough (2^28 tokens)
 for HBM bandwidth, not launch latency, to be what is measured.  Both print
-markdown tables.
+markdown tables.  `ceiling` runs the three contractions of the single-pass loss for a few
+seconds (so that the power cap, not the burst clock, sets the pace) and then the library's
+plain GEMMs (torch.matmul) on the same shapes and the same operand values for as long: what
+a tensor-core kernel without the loss epilogues reaches on this data under this cap.
 """
 import argparse
 import json
@@ -160,15 +164,143 @@ def one_chunk_sample(name="qwen3_8b", rows=16384, calls=2):
     return f"{int(st.n_sel.item())} rows of the {name} head, {calls} single-pass calls"
 
 
+def _clock_sampler():
+    import subprocess
+    try:
+        return subprocess.Popen(
+            ["nvidia-smi", "-i", str(torch.cuda.current_device()), "--query-gpu=clocks.sm,power.draw",
+             "--format=csv,noheader,nounits", "-lms", "200"], stdout=subprocess.PIPE,
+            stderr=subprocess.DEVNULL, text=True)
+    except OSError:
+        return None
+
+
+def _clock_median(proc):
+    if proc is None:
+        return float("nan"), float("nan")
+    proc.terminate()
+    out, _ = proc.communicate(timeout=10)
+    sm, pw = [], []
+    for line in out.splitlines():
+        parts = [c.strip() for c in line.split(",")]
+        try:
+            sm.append(float(parts[0]))
+            pw.append(float(parts[1]))
+        except (ValueError, IndexError):
+            continue
+    # the upper half of the samples: those taken while the loop was running
+    sm.sort()
+    pw.sort()
+    half = len(sm) // 2
+    return (statistics.median(sm[half:]) if sm else float("nan"),
+            statistics.median(pw[half:]) if pw else float("nan"))
+
+
+def ceiling(name="qwen3_8b", rows=32768, seconds=4.0):
+    """Per contraction: TFLOP/s of the loss kernels and of the library GEMM on the same
+    operands, each measured inside a loop that runs for `seconds` under the power cap."""
+    from . import nat
+    base = wl.WORKLOADS[name]
+    T = rows // base.G
+    w = wl.variant(base, P=1, sel_mode="urs", p=1.0, length_law="uniform", len_lo=T, len_hi=T)
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = NatStep(w.P, w.G, w.d, w.V, torch.bfloat16, batch["n_tot"])
+    cu = batch["cu_seqlens"]
+    st.grpo_adv(batch["rewards"])
+    st.select(cu, "urs", p=1.0)
+    st.compact(cu)
+    n = int(st.n_sel.item())
+    args = (batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+    ms_call = _time(lambda: st.loss_fwd_bwd(*args), 2)
+    calls = max(2, int(seconds * 1e3 / ms_call))
+    proc = _clock_sampler()
+    for _ in range(calls // 2):
+        st.loss_fwd_bwd(*args)
+    nat.nat_trace_begin()
+    for _ in range(calls - calls // 2):
+        st.loss_fwd_bwd(*args)
+    tr = nat.nat_trace_end()
+    torch.cuda.synchronize()
+    ours_clk = _clock_median(proc)
+    assert st.status() & ~4 == 0
+    traced = calls - calls // 2
+    flop = 2.0 * n * w.d * w.V
+    ours = {k: flop / (tr[k][0] / traced * 1e-3) / 1e12 for k in ("e", "dh", "dw")}
+
+    # the same three products by the library, chunk by chunk, on the same values
+    chunk = 8192
+    H = batch["hidden"][:n]
+    W = batch["W"]
+    Hc = H[:chunk]
+    S = (Hc @ W.t()).float()
+    E = torch.exp(S - S[:, :256].max(dim=1, keepdim=True).values).to(torch.bfloat16)
+    del S
+    Hs = (Hc.float() * (-1e-4 / E.float().sum(dim=1, keepdim=True))).to(torch.bfloat16)
+    Et = E.t()
+    Wt = W.t()
+    out_s = torch.empty(chunk, w.V, dtype=torch.bfloat16, device="cuda")
+    out_h = torch.empty(chunk, w.d, dtype=torch.bfloat16, device="cuda")
+    out_w = torch.empty(w.V, w.d, dtype=torch.bfloat16, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+
+    def lib_chunk(record):
+        if record:
+            ev[0].record()
+        torch.matmul(Hc, Wt, out=out_s)
+        if record:
+            ev[1].record()
+        torch.matmul(E, W, out=out_h)
+        if record:
+            ev[2].record()
+        torch.matmul(Et, Hs, out=out_w)
+        if record:
+            ev[3].record()
+
+    ms_chunk = _time(lambda: lib_chunk(False), 4)
+    reps = max(4, int(seconds * 1e3 / ms_chunk))
+    proc = _clock_sampler()
+    for _ in range(reps // 2):
+        lib_chunk(False)
+    sums = [0.0, 0.0, 0.0]
+    for _ in range(reps - reps // 2):
+        lib_chunk(True)
+        torch.cuda.synchronize()
+        for j in range(3):
+            sums[j] += ev[j].elapsed_time(ev[j + 1])
+    lib_clk = _clock_median(proc)
+    timed = reps - reps // 2
+    cflop = 2.0 * chunk * w.d * w.V
+    lib = {k: cflop / (sums[j] / timed * 1e-3) / 1e12 for j, k in enumerate(("e", "dh", "dw"))}
+    peaks, kind = _peaks()
+    label = {"e": "S = Hc W^T (kE: + exp, row sums, bf16 store)",
+             "dh": "dH = E W (kDh: + row factor, one-hot term)",
+             "dw": "dW += E^T Hs (kDw: fp32 accumulation into dW)"}
+    out = [f"{n} rows of the {name} head (d = {w.d}, V = {w.V}); each side looped for about "
+           f"{seconds:.0f} s, second half timed; library = torch.matmul, bf16 output, no "
+           f"accumulation; peaks {kind}: sustained {peaks['bf16_tflops_sustained']:.0f} TFLOP/s.", "",
+           "| contraction | loss kernel TFLOP/s | library GEMM TFLOP/s | ratio |", "|---|---|---|---|"]
+    for k in ("e", "dh", "dw"):
+        out.append(f"| {label[k]} | {ours[k]:.0f} | {lib[k]:.0f} | {ours[k] / lib[k]:.3f} |")
+    tot_o = 3.0 / sum(1.0 / ours[k] for k in ours)
+    tot_l = 3.0 / sum(1.0 / lib[k] for k in lib)
+    out.append(f"| all three (harmonic mean) | {tot_o:.0f} | {tot_l:.0f} | {tot_o / tot_l:.3f} |")
+    out += ["", f"SM clock / board power while looping (median of the busy samples): loss kernels "
+            f"{ours_clk[0]:.0f} MHz / {ours_clk[1]:.0f} W, library {lib_clk[0]:.0f} MHz / "
+            f"{lib_clk[1]:.0f} W."]
+    return "\n".join(out)
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["fraction", "stress", "chunk"])
+    ap.add_argument("what", choices=["fraction", "stress", "chunk", "ceiling"])
     ap.add_argument("--workload", default="qwen3_8b")
     ap.add_argument("--reps", type=int, default=2)
     ap.add_argument("--log2-tokens", type=int, default=28)
     args = ap.parse_args()
     if args.what == "chunk":
         print(one_chunk_sample(args.workload))
+    elif args.what == "ceiling":
+        print(ceiling(args.workload))
     elif args.what == "fraction":
         print(fraction_sweep(args.workload, reps=args.reps))
     else:
