@@ -7,6 +7,8 @@
 // Floating-point steps that must agree bit for bit with a plain IEEE
 // evaluation use the explicit round-to-nearest intrinsics, which the compiler
 // never contracts into fused multiply-adds.
+#include <climits>
+#include <cstdint>
 #include <mutex>
 
 #include "nat_common.cuh"
@@ -48,6 +50,51 @@ __device__ __forceinline__ int owner_of(const int32_t* __restrict__ cu, int B, i
     if ((int64_t)__ldg(cu + mid) <= n) lo = mid; else hi = mid;
   }
   return lo;
+}
+
+// First index i >= lo with cu[i] > x among cu[0..B] (B + 1 if there is none), found by a
+// whole warp: every step probes 32 positions at once, so a stream of 2^15 responses takes
+// four dependent loads instead of fifteen.  The first step probes 32 consecutive entries
+// because the answer is usually next to the hint.  All 32 lanes call it with the same
+// arguments; cu[i] <= x must hold for every i < lo.
+__device__ __forceinline__ int warp_upper_bound(const int32_t* __restrict__ cu, int B, int64_t x,
+                                                int lo) {
+  const int lane = threadIdx.x & 31;
+  int hi = B + 1;
+  int step = 1;
+  while (lo < hi) {
+    const int idx = lo + lane * step;
+    const bool gt = idx >= hi || (int64_t)__ldg(cu + idx) > x;
+    const unsigned b = __ballot_sync(0xFFFFFFFFu, gt);
+    if (b == 0u) {
+      lo += 31 * step + 1;
+    } else {
+      const int f = __ffs(b) - 1;
+      hi = min(hi, lo + f * step);
+      if (f > 0) lo += (f - 1) * step + 1;
+    }
+    step = max(1, (hi - lo + 31) / 32);
+  }
+  return lo;
+}
+
+// The searches a block makes for the responses around its token range usually end inside
+// one window of 32 consecutive cu entries placed by proportion (position / n_tot * B), so
+// one load serves them all.  cu_window loads the window (one entry per lane, +infinity
+// past cu[B]); window_first turns the ballot of a monotone predicate over it into the first
+// index where it holds, or reports a miss when that index may lie outside the window.
+__device__ __forceinline__ int64_t cu_window(const int32_t* __restrict__ cu, int B, int64_t x,
+                                             int64_t n_tot, int* w0) {
+  const int guess = (int)((x * (int64_t)B) / (n_tot > 0 ? n_tot : 1));
+  *w0 = max(0, min(guess - 8, B - 30));
+  const int idx = *w0 + (int)(threadIdx.x & 31);
+  return idx <= B ? (int64_t)__ldg(cu + idx) : INT64_MAX;
+}
+
+__device__ __forceinline__ bool window_first(unsigned ballot, int w0, int* out) {
+  if (ballot == 0u || ((ballot & 1u) != 0u && w0 > 0)) return false;
+  *out = w0 + __ffs(ballot) - 1;
+  return true;
 }
 
 // ------------------------------------------------------------ advantages
@@ -115,12 +162,46 @@ __device__ __forceinline__ int owner_between(const int32_t* __restrict__ cu, int
   return lo;
 }
 
-// One block per 4096 consecutive packed tokens, one thread per 16 of them (so a thread
-// reuses each Philox block for up to four tokens).  The mask leaves as one 16-byte store
-// per thread; pi is transposed through shared memory so that every warp store covers 512
-// contiguous bytes.
+// One block per 4096 consecutive packed tokens, one thread per 16 of them.  The mask
+// leaves as one 16-byte store per thread and pi as 16-byte stores that cover 512
+// contiguous bytes per warp.
+//
+// URS.  Token t of response i uses word (t-1) % 4 of Philox block (t-1) / 4, so 16
+// consecutive tokens of one response need four blocks when they start on a block
+// boundary and a fifth otherwise.  A thread evaluates the four blocks that start at or
+// before its first token; the up to three draws it still lacks are the first block of the
+// thread after it (same response, same alignment) and arrive by a warp shuffle, or through
+// shared memory from the next warp.  Only a thread whose successor cannot help (end of the
+// block, or a response boundary) evaluates a fifth block.  pi is a constant.
+//
+// RPC / truncation.  No draws per token; pi = (T-t+1)/(T-C+1) must be the correctly
+// rounded float32 quotient.  With y = RN(1/b) computed once per response, q0 = RN(a y),
+// r = a - q0 b (exact in an FMA) and q = RN(q0 + r y) is the correctly rounded a/b
+// (Markstein's theorem on FMA division); three operations per token instead of a division.
 constexpr int kSelBlockTokens = kSelThreads * kTokPerThread;  // 4096
 constexpr int kPiPad = kTokPerThread + 1;                     // 17: conflict-free rows
+
+__device__ __forceinline__ float div_rn_by(float a, float b, float rcp_b) {
+  const float q0 = __fmul_rn(a, rcp_b);
+  const float r = __fmaf_rn(-q0, b, a);
+  return __fmaf_rn(r, rcp_b, q0);
+}
+
+// 16 mask bits -> 16 bytes of 0/1 (bit j -> byte j).
+__device__ __forceinline__ uint4 bits_to_bytes(uint32_t bits) {
+  constexpr uint32_t kSpread = 0x00204081u;  // 1 + 2^7 + 2^14 + 2^21
+  uint4 v;
+  v.x = ((bits & 0xFu) * kSpread) & 0x01010101u;
+  v.y = (((bits >> 4) & 0xFu) * kSpread) & 0x01010101u;
+  v.z = (((bits >> 8) & 0xFu) * kSpread) & 0x01010101u;
+  v.w = (((bits >> 12) & 0xFu) * kSpread) & 0x01010101u;
+  return v;
+}
+
+__device__ __forceinline__ uint32_t philox_below(const Philox4& r, uint64_t thr) {
+  return ((uint64_t)r.x < thr ? 1u : 0u) | ((uint64_t)r.y < thr ? 2u : 0u) |
+         ((uint64_t)r.z < thr ? 4u : 0u) | ((uint64_t)r.w < thr ? 8u : 0u);
+}
 
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
@@ -128,72 +209,167 @@ select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
               float* __restrict__ pi) {
   __shared__ float pi_s[kSelThreads * kPiPad];
   __shared__ int range_s[2];
+  __shared__ int edge_tag_s[kSelThreads / 32 + 1];
+  __shared__ uint32_t edge_nib_s[kSelThreads / 32 + 1];
   const int64_t nb0 = (int64_t)blockIdx.x * kSelBlockTokens;
   const int cnt_block = (int)min((int64_t)kSelBlockTokens, n_tot - nb0);
-  if (threadIdx.x == 0) {
-    range_s[0] = owner_of(cu, B, nb0);
-    range_s[1] = owner_of(cu, B, nb0 + cnt_block - 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp == 0) {  // responses that own the block's first and last token
+    const int64_t last = nb0 + cnt_block - 1;
+    int w0, ub0 = 0, ub1 = 0;
+    const int64_t v = cu_window(cu, B, nb0, n_tot, &w0);
+    const bool hit = window_first(__ballot_sync(0xFFFFFFFFu, v > nb0), w0, &ub0) &&
+                     window_first(__ballot_sync(0xFFFFFFFFu, v > last), w0, &ub1);
+    if (!hit) {
+      ub0 = warp_upper_bound(cu, B, nb0, 0);
+      ub1 = warp_upper_bound(cu, B, last, ub0);
+    }
+    const int r0 = ub0 - 1, r1 = ub1 - 1;
+    if (lane == 0) {
+      range_s[0] = r0;
+      range_s[1] = r1;
+      edge_tag_s[kSelThreads / 32] = -1;  // nobody follows the last warp
+    }
   }
   __syncthreads();
   const int64_t n0 = nb0 + (int64_t)threadIdx.x * kTokPerThread;
-  if (n0 < n_tot) {
-    const int cnt = (int)min((int64_t)kTokPerThread, n_tot - n0);
-    int i = owner_between(cu, range_s[0], range_s[1], n0);
-    int64_t start = cu[i], end = cu[i + 1];
-    int L = 0, C = 0;
-    float den = 1.f;
-    auto enter_response = [&]() {
-      if (c.mode != NAT_SEL_URS) {
-        L = cut_len[i];
-        const int T = (int)(end - start);
-        C = (c.mode == NAT_SEL_RPC) ? min(max(c.min_cut, 1), T) : T;
-        den = (float)(T - C + 1);
-      }
-    };
-    enter_response();
-    uint32_t cached_blk = 0xFFFFFFFFu;
-    int cached_resp = -1;
-    Philox4 rnd = {0, 0, 0, 0};
+  const bool active = n0 < n_tot;
+  const int cnt = active ? (int)min((int64_t)kTokPerThread, n_tot - n0) : 0;
+  int i = 0;
+  int64_t start = 0, end = 0;
+  if (active) {
+    i = owner_between(cu, range_s[0], range_s[1], n0);
+    start = cu[i];
+    end = cu[i + 1];
+  }
+  // the whole 16-token span lies inside response i
+  const bool inside = active && cnt == kTokPerThread && n0 + kTokPerThread <= end;
+  uint32_t bits = 0;
 
-    alignas(16) uint8_t m[kTokPerThread];
-    float* pr = pi_s + threadIdx.x * kPiPad;
+  if (c.mode == NAT_SEL_URS) {
+    const uint32_t t0 = (uint32_t)(n0 - start);  // (position - 1) of the first token
+    const uint32_t sh = t0 & 3u;
+    uint32_t low = 0;                            // draws of blocks blk0 .. blk0+3, bit 4q+word
+    if (inside) {
+      const uint32_t blk0 = t0 >> 2;
 #pragma unroll
-    for (int j = 0; j < kTokPerThread; ++j) {
-      m[j] = 0;
-      float pv = 0.f;
-      if (j < cnt) {
-        const int64_t n = n0 + j;
-        while (n >= end) {  // skips empty responses too
-          ++i;
-          start = end;
-          end = cu[i + 1];
-          if (n < end) enter_response();
-        }
-        const uint32_t t0 = (uint32_t)(n - start);  // t - 1
-        if (c.mode == NAT_SEL_URS) {
-          const uint32_t blk = t0 >> 2;
+      for (int q = 0; q < 4; ++q)
+        low |= philox_below(philox4x32_10(blk0 + q, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1), c.thr)
+               << (4 * q);
+    }
+    const int tag = inside ? i : -1;
+    if (lane == 0) {
+      edge_tag_s[warp] = tag;
+      edge_nib_s[warp] = low & 0xFu;
+    }
+    int next_tag = __shfl_down_sync(0xFFFFFFFFu, tag, 1);
+    uint32_t next_nib = __shfl_down_sync(0xFFFFFFFFu, low, 1) & 0xFu;
+    __syncthreads();
+    if (lane == 31) {
+      next_tag = edge_tag_s[warp + 1];
+      next_nib = edge_nib_s[warp + 1];
+    }
+    if (inside) {
+      if (sh != 0u && next_tag != i)
+        next_nib = philox_below(
+            philox4x32_10((t0 >> 2) + 4u, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1), c.thr);
+      bits = ((low | (next_nib << 16)) >> sh) & 0xFFFFu;
+      *reinterpret_cast<uint4*>(mask + n0) = bits_to_bytes(bits);
+    } else if (active) {
+      // a span that crosses a response boundary or the end of the stream: token by token
+      uint32_t cached_blk = 0xFFFFFFFFu;
+      int cached_resp = -1;
+      Philox4 rnd = {0, 0, 0, 0};
+      alignas(16) uint8_t m[kTokPerThread];
+#pragma unroll
+      for (int j = 0; j < kTokPerThread; ++j) {
+        m[j] = 0;
+        if (j < cnt) {
+          const int64_t n = n0 + j;
+          while (n >= end) {  // skips empty responses too
+            ++i;
+            start = end;
+            end = cu[i + 1];
+          }
+          const uint32_t tj = (uint32_t)(n - start);
+          const uint32_t blk = tj >> 2;
           if (blk != cached_blk || i != cached_resp) {
             rnd = philox4x32_10(blk, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1);
             cached_blk = blk;
             cached_resp = i;
           }
-          const uint32_t lane = t0 & 3u;
-          const uint32_t x = lane == 0 ? rnd.x : lane == 1 ? rnd.y : lane == 2 ? rnd.z : rnd.w;
+          const uint32_t word = tj & 3u;
+          const uint32_t x = word == 0 ? rnd.x : word == 1 ? rnd.y : word == 2 ? rnd.z : rnd.w;
           m[j] = ((uint64_t)x < c.thr) ? 1 : 0;
-          pv = c.pi_urs;
-        } else {
-          const int t = (int)t0 + 1;
-          m[j] = (t <= L) ? 1 : 0;
-          const int T = (int)(end - start);
-          pv = (t <= C) ? 1.f : __fdiv_rn((float)(T - t + 1), den);
         }
       }
-      pr[j] = pv;
+      if (cnt == kTokPerThread) {
+        *reinterpret_cast<uint4*>(mask + n0) = *reinterpret_cast<const uint4*>(m);
+      } else {
+        for (int j = 0; j < cnt; ++j) mask[n0 + j] = m[j];
+      }
     }
-    if (cnt == kTokPerThread) {
-      *reinterpret_cast<uint4*>(mask + n0) = *reinterpret_cast<const uint4*>(m);
+    // pi is the same for every token
+    if (cnt_block == kSelBlockTokens) {
+      const float4 v = make_float4(c.pi_urs, c.pi_urs, c.pi_urs, c.pi_urs);
+#pragma unroll
+      for (int k = 0; k < kTokPerThread / 4; ++k)
+        *reinterpret_cast<float4*>(pi + nb0 + (int64_t)(k * kSelThreads + threadIdx.x) * 4) = v;
     } else {
-      for (int j = 0; j < cnt; ++j) mask[n0 + j] = m[j];
+      for (int e = threadIdx.x; e < cnt_block; e += kSelThreads) pi[nb0 + e] = c.pi_urs;
+    }
+    return;
+  }
+
+  // ---- RPC / deterministic truncation
+  if (active) {
+    int L = 0, C = 0;
+    float den = 1.f, rden = 1.f;
+    auto enter_response = [&]() {
+      L = cut_len[i];
+      const int T = (int)(end - start);
+      C = (c.mode == NAT_SEL_RPC) ? min(max(c.min_cut, 1), T) : T;
+      den = (float)(T - C + 1);
+      rden = __frcp_rn(den);
+    };
+    enter_response();
+    float* pr = pi_s + threadIdx.x * kPiPad;
+    if (inside) {
+      const int T = (int)(end - start);
+      const int t_first = (int)(n0 - start) + 1;
+#pragma unroll
+      for (int j = 0; j < kTokPerThread; ++j) {
+        const int t = t_first + j;
+        bits |= (t <= L ? 1u : 0u) << j;
+        pr[j] = (t <= C) ? 1.f : div_rn_by((float)(T - t + 1), den, rden);
+      }
+      *reinterpret_cast<uint4*>(mask + n0) = bits_to_bytes(bits);
+    } else {
+      alignas(16) uint8_t m[kTokPerThread];
+#pragma unroll
+      for (int j = 0; j < kTokPerThread; ++j) {
+        m[j] = 0;
+        float pv = 0.f;
+        if (j < cnt) {
+          const int64_t n = n0 + j;
+          while (n >= end) {  // skips empty responses too
+            ++i;
+            start = end;
+            end = cu[i + 1];
+            if (n < end) enter_response();
+          }
+          const int t = (int)(n - start) + 1;
+          const int T = (int)(end - start);
+          m[j] = (t <= L) ? 1 : 0;
+          pv = (t <= C) ? 1.f : div_rn_by((float)(T - t + 1), den, rden);
+        }
+        pr[j] = pv;
+      }
+      if (cnt == kTokPerThread) {
+        *reinterpret_cast<uint4*>(mask + n0) = *reinterpret_cast<const uint4*>(m);
+      } else {
+        for (int j = 0; j < cnt; ++j) mask[n0 + j] = m[j];
+      }
     }
   }
   __syncthreads();
@@ -294,6 +470,7 @@ move_rows_kernel(const uint4* __restrict__ src, int64_t row_vec,
 // falls inside the chunk.
 constexpr int kCmpThreads = 256;
 constexpr int kChunk = kCmpThreads * kTokPerThread;  // 4096 tokens
+constexpr int kCountChunks = 8;                      // chunks per block of the counting pass
 
 __device__ __forceinline__ uint32_t load_mask_bits(const uint8_t* __restrict__ mask, int64_t n0,
                                                    int64_t n_tot) {
@@ -302,10 +479,11 @@ __device__ __forceinline__ uint32_t load_mask_bits(const uint8_t* __restrict__ m
     const uint4 v = __ldg(reinterpret_cast<const uint4*>(mask + n0));
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-#pragma unroll
-      for (int b = 0; b < 4; ++b)
-        if ((w[q] >> (8 * b)) & 0xFFu) bits |= 1u << (4 * q + b);
+    for (int q = 0; q < 4; ++q) {
+      // byte != 0 -> its bit 7 set -> gathered into bits 0..3 (a multiply collects them)
+      const uint32_t nz = ((w[q] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu | w[q]) & 0x80808080u;
+      bits |= (((nz >> 7) * 0x01020408u) >> 24 & 0xFu) << (4 * q);
+    }
   } else {
     for (int j = 0; j < kTokPerThread; ++j)
       if (n0 + j < n_tot && mask[n0 + j] != 0) bits |= 1u << j;
@@ -313,65 +491,98 @@ __device__ __forceinline__ uint32_t load_mask_bits(const uint8_t* __restrict__ m
   return bits;
 }
 
+// Each block counts kCountChunks consecutive chunks: that many independent 16-byte loads
+// per thread are in flight at once.
 __global__ void __launch_bounds__(kCmpThreads)
-compact_count_kernel(const uint8_t* __restrict__ mask, int64_t n_tot,
+compact_count_kernel(const uint8_t* __restrict__ mask, int64_t n_tot, int n_chunks,
                      int32_t* __restrict__ chunk_count) {
-  __shared__ int warp_sum[kCmpThreads / 32];
-  const int64_t n0 = (int64_t)blockIdx.x * kChunk + (int64_t)threadIdx.x * kTokPerThread;
-  int c = (n0 < n_tot) ? __popc(load_mask_bits(mask, n0, n_tot)) : 0;
-  c = __reduce_add_sync(0xFFFFFFFFu, c);
-  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = c;
+  __shared__ int warp_sum[kCountChunks][kCmpThreads / 32];
+  const int chunk_first = blockIdx.x * kCountChunks;
+  int c[kCountChunks];
+#pragma unroll
+  for (int q = 0; q < kCountChunks; ++q) {
+    const int64_t n0 = (int64_t)(chunk_first + q) * kChunk + (int64_t)threadIdx.x * kTokPerThread;
+    c[q] = (n0 < n_tot) ? __popc(load_mask_bits(mask, n0, n_tot)) : 0;
+  }
+#pragma unroll
+  for (int q = 0; q < kCountChunks; ++q) {
+    const int r = __reduce_add_sync(0xFFFFFFFFu, c[q]);
+    if ((threadIdx.x & 31) == 0) warp_sum[q][threadIdx.x >> 5] = r;
+  }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    int s = 0;
-    for (int w = 0; w < kCmpThreads / 32; ++w) s += warp_sum[w];
-    chunk_count[blockIdx.x] = s;
+  if (threadIdx.x < kCountChunks && chunk_first + (int)threadIdx.x < n_chunks) {
+    int t = 0;
+    for (int w = 0; w < kCmpThreads / 32; ++w) t += warp_sum[threadIdx.x][w];
+    chunk_count[chunk_first + threadIdx.x] = t;
   }
 }
 
 // Exclusive scan of the chunk counts by a single block (in place), total to
-// chunk_count[n_chunks], n_sel and sel_offsets[B].
+// chunk_count[n_chunks], n_sel and sel_offsets[B].  Tiles of 4096 counts: every thread
+// takes four consecutive counts with one 16-byte load (the next tile's load is issued
+// before this tile's barrier), the warps scan by shuffles and meet once per tile.
 __global__ void __launch_bounds__(1024)
 compact_scan_kernel(int32_t* __restrict__ chunk_count, int n_chunks, int32_t* __restrict__ n_sel,
                     int32_t* __restrict__ sel_offsets, int B) {
-  __shared__ int warp_tot[32];
-  __shared__ int carry_s;
-  if (threadIdx.x == 0) carry_s = 0;
-  __syncthreads();
-  for (int base = 0; base < n_chunks; base += 1024) {
-    const int idx = base + threadIdx.x;
-    const int v = idx < n_chunks ? chunk_count[idx] : 0;
-    int incl = v;
+  __shared__ int warp_tot[2][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n_tiles = (n_chunks + 4095) / 4096;
+  auto load4 = [&](int tile) {
+    const int k = tile * 4096 + (int)threadIdx.x * 4;
+    int4 v = make_int4(0, 0, 0, 0);
+    if (k < n_chunks) v = *reinterpret_cast<const int4*>(chunk_count + k);  // padded allocation
+    if (k + 1 >= n_chunks) v.y = 0;
+    if (k + 2 >= n_chunks) v.z = 0;
+    if (k + 3 >= n_chunks) v.w = 0;
+    return v;
+  };
+  int carry = 0;
+  int4 cur = n_tiles > 0 ? load4(0) : make_int4(0, 0, 0, 0);
+  for (int tile = 0; tile < n_tiles; ++tile) {
+    const int4 nxt = tile + 1 < n_tiles ? load4(tile + 1) : make_int4(0, 0, 0, 0);
+    const int sum = cur.x + cur.y + cur.z + cur.w;
+    int incl = sum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-      if ((threadIdx.x & 31) >= o) incl += up;
+      if (lane >= o) incl += up;
     }
-    if ((threadIdx.x & 31) == 31) warp_tot[threadIdx.x >> 5] = incl;
+    int* tot = warp_tot[tile & 1];
+    if (lane == 31) tot[warp] = incl;
     __syncthreads();
-    if (threadIdx.x < 32) {
-      int w = warp_tot[threadIdx.x];
+    // every warp scans the 32 warp totals itself
+    const int wt = tot[lane];
+    int wincl = wt;
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int up = __shfl_up_sync(0xFFFFFFFFu, w, o);
-        if (threadIdx.x >= o) w += up;
-      }
-      warp_tot[threadIdx.x] = w;  // inclusive over warps
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xFFFFFFFFu, wincl, o);
+      if (lane >= o) wincl += up;
     }
-    __syncthreads();
-    const int carry = carry_s;
-    const int warp_excl = (threadIdx.x >> 5) ? warp_tot[(threadIdx.x >> 5) - 1] : 0;
-    if (idx < n_chunks) chunk_count[idx] = carry + warp_excl + incl - v;
-    __syncthreads();
-    if (threadIdx.x == 0) carry_s = carry + warp_tot[31];
-    __syncthreads();
+    const int tile_total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
+    const int warp_excl = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp);
+    const int e0 = carry + warp_excl + incl - sum;
+    const int k = tile * 4096 + (int)threadIdx.x * 4;
+    if (k + 3 < n_chunks) {
+      *reinterpret_cast<int4*>(chunk_count + k) =
+          make_int4(e0, e0 + cur.x, e0 + cur.x + cur.y, e0 + cur.x + cur.y + cur.z);
+    } else {
+      if (k < n_chunks) chunk_count[k] = e0;
+      if (k + 1 < n_chunks) chunk_count[k + 1] = e0 + cur.x;
+      if (k + 2 < n_chunks) chunk_count[k + 2] = e0 + cur.x + cur.y;
+    }
+    carry += tile_total;
+    cur = nxt;
   }
   if (threadIdx.x == 0) {
-    chunk_count[n_chunks] = carry_s;
-    *n_sel = carry_s;
-    sel_offsets[B] = carry_s;
+    chunk_count[n_chunks] = carry;
+    *n_sel = carry;
+    sel_offsets[B] = carry;
   }
 }
+
+// Staging index of output slot k: one spare slot after every 32 keeps both the writes
+// (threads 8 or 16 slots apart) and the reads (consecutive slots) free of bank conflicts.
+__device__ __forceinline__ int skew(int k) { return k + (k >> 5); }
 
 __global__ void __launch_bounds__(kCmpThreads)
 compact_write_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
@@ -381,17 +592,33 @@ compact_write_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
   __shared__ int warp_tot[kCmpThreads / 32];
   __shared__ int thread_excl[kCmpThreads];
   __shared__ uint32_t thread_bits[kCmpThreads];
-  __shared__ int32_t idx_s[kChunk];
-  __shared__ int32_t resp_s[kChunk];
-  __shared__ int range_s[2];
+  __shared__ int32_t idx_s[kChunk + kChunk / 32];
+  __shared__ int32_t resp_s[kChunk + kChunk / 32];
+  __shared__ int range_s[3];
   const int64_t chunk0 = (int64_t)blockIdx.x * kChunk;
-  if (threadIdx.x == 0) {  // responses that own the chunk's first and last token
-    const int64_t last = min(chunk0 + (int64_t)kChunk, n_tot) - 1;
-    range_s[0] = owner_of(cu, B, chunk0);
-    range_s[1] = owner_of(cu, B, last);
-  }
+  const int64_t chunk_end = min(chunk0 + (int64_t)kChunk, n_tot);
   const int64_t n0 = chunk0 + (int64_t)threadIdx.x * kTokPerThread;
   const uint32_t bits = (n0 < n_tot) ? load_mask_bits(mask, n0, n_tot) : 0u;
+  const int base = chunk_offset[blockIdx.x];
+  if (threadIdx.x < 32) {
+    // first response whose start lies in this chunk, and the responses that own the
+    // chunk's first and last token
+    int w0, first_in = 0, ub0 = 0, ub1 = 0;
+    const int64_t v = cu_window(cu, B, chunk0, n_tot, &w0);
+    const bool hit = window_first(__ballot_sync(0xFFFFFFFFu, v >= chunk0), w0, &first_in) &&
+                     window_first(__ballot_sync(0xFFFFFFFFu, v > chunk0), w0, &ub0) &&
+                     window_first(__ballot_sync(0xFFFFFFFFu, v > chunk_end - 1), w0, &ub1);
+    if (!hit) {
+      first_in = warp_upper_bound(cu, B, chunk0 - 1, 0);
+      ub0 = warp_upper_bound(cu, B, chunk0, first_in);
+      ub1 = warp_upper_bound(cu, B, chunk_end - 1, ub0);
+    }
+    if (threadIdx.x == 0) {
+      range_s[0] = ub0 - 1;
+      range_s[1] = ub1 - 1;
+      range_s[2] = first_in;
+    }
+  }
   const int c = __popc(bits);
   int incl = c;
 #pragma unroll
@@ -403,24 +630,42 @@ compact_write_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
   __syncthreads();
   int warp_excl = 0;
   for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) warp_excl += warp_tot[w];
-  const int base = chunk_offset[blockIdx.x];
   const int excl = base + warp_excl + incl - c;  // selected tokens before n0
   thread_excl[threadIdx.x] = excl;
   thread_bits[threadIdx.x] = bits;
-  __syncthreads();
 
   // The chunk's selected tokens are consecutive in the output lists: stage them in
-  // shared memory, then write them out with fully coalesced stores.
+  // shared memory, then write them out with coalesced 16-byte stores.  A chunk that lies
+  // inside one response (the usual case for long responses) has a constant owner and
+  // stages the indices only.
+  const int r_first = range_s[0];
+  const bool one_owner = (r_first == range_s[1]);
   if (bits != 0u) {
-    int i = owner_between(cu, range_s[0], range_s[1], n0);
-    int64_t end = cu[i + 1];
     int k = excl - base;
-    for (int j = 0; j < kTokPerThread; ++j) {
-      if ((bits >> j) & 1u) {
+    int i = r_first;
+    int64_t end = INT64_MAX;
+    if (!one_owner) {
+      i = owner_between(cu, r_first, range_s[1], n0);
+      end = cu[i + 1];
+    }
+    if (n0 + kTokPerThread <= end) {  // the thread's 16 tokens have one owner
+#pragma unroll
+      for (int j = 0; j < kTokPerThread; ++j) {
+        if ((bits >> j) & 1u) {
+          idx_s[skew(k)] = (int32_t)(n0 + j);
+          if (!one_owner) resp_s[skew(k)] = i;
+          ++k;
+        }
+      }
+    } else {
+      uint32_t rest = bits;
+      while (rest != 0u) {
+        const int j = __ffs(rest) - 1;
+        rest &= rest - 1u;
         const int64_t n = n0 + j;
         while (n >= end) end = cu[++i + 1];
-        idx_s[k] = (int32_t)n;
-        resp_s[k] = i;
+        idx_s[skew(k)] = (int32_t)n;
+        resp_s[skew(k)] = i;
         ++k;
       }
     }
@@ -429,26 +674,45 @@ compact_write_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
   {
     int total = 0;
     for (int w = 0; w < kCmpThreads / 32; ++w) total += warp_tot[w];
-    for (int e = threadIdx.x; e < total; e += kCmpThreads) {
-      const int64_t k = (int64_t)base + e;
-      if (k < cap) {
-        sel_idx[k] = idx_s[e];
-        sel_resp[k] = resp_s[e];
+    const bool vec_ok = (int64_t)base + total <= cap &&
+                        ((reinterpret_cast<uintptr_t>(sel_idx) |
+                          reinterpret_cast<uintptr_t>(sel_resp)) & 15u) == 0;
+    if (vec_ok) {
+      // slots [head, head + 4 * groups) start on a 16-byte boundary of the output lists
+      const int head = min(total, (4 - (base & 3)) & 3);
+      const int groups = (total - head) / 4;
+      for (int g = threadIdx.x; g < groups; g += kCmpThreads) {
+        const int e = head + 4 * g;
+        const int4 v = make_int4(idx_s[skew(e)], idx_s[skew(e + 1)], idx_s[skew(e + 2)],
+                                 idx_s[skew(e + 3)]);
+        const int4 r = one_owner ? make_int4(r_first, r_first, r_first, r_first)
+                                 : make_int4(resp_s[skew(e)], resp_s[skew(e + 1)],
+                                             resp_s[skew(e + 2)], resp_s[skew(e + 3)]);
+        *reinterpret_cast<int4*>(sel_idx + base + e) = v;
+        *reinterpret_cast<int4*>(sel_resp + base + e) = r;
+      }
+      const int done = head + 4 * groups;
+      const int rest_n = head + (total - done);  // slots before the first and after the last group
+      if ((int)threadIdx.x < rest_n) {
+        const int e = (int)threadIdx.x < head ? (int)threadIdx.x : done + ((int)threadIdx.x - head);
+        sel_idx[base + e] = idx_s[skew(e)];
+        sel_resp[base + e] = one_owner ? r_first : resp_s[skew(e)];
+      }
+    } else {
+      for (int e = threadIdx.x; e < total; e += kCmpThreads) {
+        const int64_t k = (int64_t)base + e;
+        if (k < cap) {
+          sel_idx[k] = idx_s[skew(e)];
+          sel_resp[k] = one_owner ? r_first : resp_s[skew(e)];
+        }
       }
     }
   }
 
   // Per-response offsets: every i with cu[i] inside this chunk (the last chunk
   // also takes the boundaries equal to n_tot).  sel_offsets[B] is the scan's.
-  const int64_t chunk_end = min(chunk0 + (int64_t)kChunk, n_tot);
   const bool last = (chunk_end == n_tot);
-  // first i with cu[i] >= chunk0
-  int lo = 0, hi = B;  // search in [0, B]
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if ((int64_t)cu[mid] < chunk0) lo = mid + 1; else hi = mid;
-  }
-  for (int i = lo + threadIdx.x; i < B; i += kCmpThreads) {
+  for (int i = range_s[2] + threadIdx.x; i < B; i += kCmpThreads) {
     const int64_t n = cu[i];
     if (n > chunk_end || (n == chunk_end && !last)) break;
     if (n == n_tot) {
@@ -631,7 +895,8 @@ int nat_compact(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8
   int32_t* chunk_count = reinterpret_cast<int32_t*>(workspace);
   const int n_chunks = (int)((n_tot + kChunk - 1) / kChunk);
   if (n_chunks > 0) {
-    compact_count_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(mask, n_tot, chunk_count);
+    compact_count_kernel<<<(n_chunks + kCountChunks - 1) / kCountChunks, kCmpThreads, 0, stream>>>(
+        mask, n_tot, n_chunks, chunk_count);
     NAT_LAUNCH_CHECK("compact_count_kernel");
   }
   compact_scan_kernel<<<1, 1024, 0, stream>>>(chunk_count, n_chunks, n_sel, sel_offsets, B);
@@ -718,7 +983,8 @@ int nat_compact_static(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, cons
   // by a previous call needs clearing.
   const int n_chunks = (int)((n_tot + kChunk - 1) / kChunk);
   if (n_chunks > 0) {
-    compact_count_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(mask, n_tot, chunk_count);
+    compact_count_kernel<<<(n_chunks + kCountChunks - 1) / kCountChunks, kCmpThreads, 0, stream>>>(
+        mask, n_tot, n_chunks, chunk_count);
     NAT_LAUNCH_CHECK("compact_count_kernel");
   }
   compact_scan_kernel<<<1, 1024, 0, stream>>>(chunk_count, n_chunks, n_sel, sel_offsets, B);
