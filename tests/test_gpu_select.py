@@ -76,6 +76,46 @@ def test_edge_cases():
     _select_compact([32768, 9], "rpc", 1, 2, seed=9, min_cut=1)
 
 
+def test_rpc_every_length_up_to_4096():
+    # every denominator T - C + 1 <= 4096 with every numerator: the kernel forms pi by an FMA
+    # sequence instead of a division and must still give the correctly rounded quotient
+    T = np.random.default_rng(0).permutation(np.arange(1, 4097))
+    _select_compact(T, "rpc", 512, 8, seed=3, min_cut=1)
+
+
+def test_rpc_pi_is_the_rounded_quotient_for_every_length_up_to_32768():
+    # all 5.4e8 quotients (T-t+1)/T with T <= 32768 (the longest response of the workloads)
+    # against numpy's float32 division, which is what the oracle's definition of pi is
+    Tmax = 32768
+    T = np.arange(1, Tmax + 1, dtype=np.int64)
+    cu = np.concatenate([[0], np.cumsum(T)])
+    n_tot, B = int(cu[-1]), Tmax
+    mask = torch.empty(n_tot, dtype=torch.uint8, device="cuda")
+    pi = torch.empty(n_tot, dtype=torch.float32, device="cuda")
+    cut = torch.empty(B, dtype=torch.int32, device="cuda")
+    nat.nat_select(nat.select_params("rpc", min_cut=1, seed=3), B,
+                   torch.from_numpy(cu.astype(np.int32)).cuda(), n_tot, mask, pi, cut)
+    torch.cuda.synchronize()
+    pi_h, mask_h, cut_h = pi.cpu().numpy(), mask.cpu().numpy(), cut.cpu().numpy()
+    del mask, pi
+    for i in range(B):
+        Ti = int(T[i])
+        t = np.arange(1, Ti + 1, dtype=np.int64)
+        ref = (Ti - t + 1).astype(np.float32) / np.float32(Ti)
+        assert np.array_equal(pi_h[cu[i]:cu[i + 1]].view(np.uint32), ref.view(np.uint32)), Ti
+        assert np.array_equal(mask_h[cu[i]:cu[i + 1]], (t <= cut_h[i]).astype(np.uint8)), Ti
+        assert 1 <= cut_h[i] <= Ti
+
+
+def test_skewed_lengths_miss_the_proportional_window():
+    # one very long response among many short ones: the blocks' proportional guess of the
+    # owning response is far off, so the general search runs
+    T = [3] * 500 + [40000] + [5] * 300 + [0] * 40 + [9000] + [2] * 182
+    assert len(T) == 1024
+    for mode in ("urs", "rpc", "det"):
+        _select_compact(T, mode, 128, 8, seed=11, min_cut=4)
+
+
 def test_capacity_smaller_than_selection():
     n = _select_compact([300, 200, 100, 50], "urs", 2, 2, seed=1, p=0.9, cap=64)
     assert n > 64
