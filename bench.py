@@ -178,11 +178,16 @@ def run_ours(args, w):
     cu = batch["cu_seqlens"]
     sel = dict(mode=w.sel_mode, p=w.p, min_cut=w.min_cut, beta=w.beta, seed=seed)
 
+    def exchange():
+        if args.allreduce_dw and world > 1:
+            sharding.allreduce_grads(st.loss, st.dW)
+
     def step(b, offset):
         st.grpo_adv(b["rewards"])
         st.select(cu, offset=offset, **sel)
         st.compact(cu)
         st.loss_fwd_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
+        exchange()
 
     def sync_all():
         torch.cuda.synchronize()
@@ -196,6 +201,7 @@ def run_ours(args, w):
         st.compact(cu)
         st.loss_fwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
         st.loss_bwd(b["hidden"], b["W"], b["targets"], b["old_logp"], cu)
+        exchange()
 
     main_step = step if args.route == "single" else step_two_pass
     for i in range(args.warmup):
@@ -227,6 +233,7 @@ def run_ours(args, w):
             ev[i][1].record()
             st.loss_bwd(batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
         ev[i][2].record()
+        exchange()
     t_end.record()
     sync_all()
     clocks = sampler.stop() if rank == 0 else None
@@ -362,7 +369,9 @@ def run_ours(args, w):
                              else "two pass (nat_policy_loss_fwd, nat_policy_loss_bwd)"),
                    "n_tot_per_gpu": n_tot, "n_sel_per_step_per_gpu": n_step,
                    "l2": "inputs larger than L2 (hidden and W_lm are GBs); no flush needed",
-                   "parallelism": f"dp{world} (independent batches, no collective)"},
+                   "parallelism": (f"dp{world} (independent batches, loss and dW all-reduced "
+                                   "every step)" if args.allreduce_dw and world > 1 else
+                                   f"dp{world} (independent batches, no collective)")},
         "tflops_counted": step_tflops,
         "tflops_executed": executed / (step_ms * 1e-3) / 1e12,
         "frac_of_peak_counted": {
@@ -410,7 +419,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen3_8b")
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--ref-rows", type=int, default=16)
+    ap.add_argument("--ref-rows", type=int, default=128,
+                    help="selected rows the fp64 oracle evaluates per timed sample (about 12 s on 16 cores)")
+    ap.add_argument("--allreduce-dw", action="store_true",
+                    help="N > 1: sum loss and dW over the ranks inside every step (the exchange of "
+                         "a data-parallel trainer); off by default: ranks then run independent "
+                         "batches with no collective")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-other-route", action="store_true",
                     help="do not also time the route that was not selected")

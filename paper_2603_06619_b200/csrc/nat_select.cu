@@ -41,17 +41,6 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
   return {c0, c1, c2, c3};
 }
 
-// Largest i with cu[i] <= n among responses that are not empty at n, i.e. the
-// response that owns packed token n (cu is non-decreasing, cu[B] > n).
-__device__ __forceinline__ int owner_of(const int32_t* __restrict__ cu, int B, int64_t n) {
-  int lo = 0, hi = B;  // invariant: cu[lo] <= n < cu[hi]
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if ((int64_t)__ldg(cu + mid) <= n) lo = mid; else hi = mid;
-  }
-  return lo;
-}
-
 // First index i >= lo with cu[i] > x among cu[0..B] (B + 1 if there is none), found by a
 // whole warp: every step probes 32 positions at once, so a stream of 2^15 responses takes
 // four dependent loads instead of fifteen.  The first step probes 32 consecutive entries
@@ -395,10 +384,28 @@ __global__ void __launch_bounds__(kSelThreads)
 select_survival_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
                        const float* __restrict__ surv, uint8_t* __restrict__ mask,
                        int32_t* __restrict__ cut_len) {
-  const int64_t n0 = ((int64_t)blockIdx.x * kSelThreads + threadIdx.x) * kTokPerThread;
+  __shared__ int range_s[2];
+  const int64_t nb0 = (int64_t)blockIdx.x * kSelBlockTokens;
+  if (threadIdx.x < 32) {  // responses that own the block's first and last token
+    const int64_t last = min(nb0 + (int64_t)kSelBlockTokens, n_tot) - 1;
+    int w0, ub0 = 0, ub1 = 0;
+    const int64_t v = cu_window(cu, B, nb0, n_tot, &w0);
+    const bool hit = window_first(__ballot_sync(0xFFFFFFFFu, v > nb0), w0, &ub0) &&
+                     window_first(__ballot_sync(0xFFFFFFFFu, v > last), w0, &ub1);
+    if (!hit) {
+      ub0 = warp_upper_bound(cu, B, nb0, 0);
+      ub1 = warp_upper_bound(cu, B, last, ub0);
+    }
+    if (threadIdx.x == 0) {
+      range_s[0] = ub0 - 1;
+      range_s[1] = ub1 - 1;
+    }
+  }
+  __syncthreads();
+  const int64_t n0 = nb0 + (int64_t)threadIdx.x * kTokPerThread;
   if (n0 >= n_tot) return;
   const int cnt = (int)min((int64_t)kTokPerThread, n_tot - n0);
-  int i = owner_of(cu, B, n0);
+  int i = owner_between(cu, range_s[0], range_s[1], n0);
   int64_t start = cu[i], end = cu[i + 1];
   auto draw = [&]() {
     const Philox4 r = philox4x32_10(0u, (uint32_t)i, 2u, c.off_lo, c.k0, c.k1);

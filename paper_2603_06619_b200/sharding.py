@@ -27,6 +27,28 @@ def rank_seed(seed, rank):
     return seed + rank
 
 
+def allreduce_grads(loss, dW, bucket_elems=64 << 20, wait=True):
+    """Sum `loss` (1 element) and `dW` ([V, d] float32) over the data-parallel ranks, in place.
+
+    This is the one exchange of a data-parallel step: every rank computed its responses'
+    share with the GLOBAL batch size in its weights, so the sums are the job's loss and
+    gradient.  dW goes out in buckets (one collective each, issued asynchronously on the
+    process group's stream) so that a caller that passes wait=False can overlap the tail of
+    its own work with them; it gets the handles to wait on.  A single process is a no-op.
+    """
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return []
+    flat = dW.reshape(-1)
+    handles = [dist.all_reduce(flat[lo:lo + bucket_elems], async_op=True)
+               for lo in range(0, flat.numel(), bucket_elems)]
+    handles.append(dist.all_reduce(loss, async_op=True))
+    if wait:
+        for h in handles:
+            h.wait()
+        return []
+    return handles
+
+
 def aggregate_timing(elapsed_ms, units, device=None):
     """(max over ranks of each elapsed time, sum over ranks of the units processed).
 

@@ -56,8 +56,10 @@ def _worker(rank, world, port, out_dir):
 
     loss = torch.tensor([out["loss"]], dtype=torch.float64)
     dW = torch.from_numpy(out["dW"].copy())
-    dist.all_reduce(loss)
-    dist.all_reduce(dW)
+    handles = sharding.allreduce_grads(loss, dW, bucket_elems=1000, wait=False)   # several buckets
+    assert len(handles) == -(-dW.numel() // 1000) + 1
+    for h in handles:
+        h.wait()
     times, units = sharding.aggregate_timing([10.0 + rank, 5.0 - rank], n)
     if rank == 0:
         si, sr, _, n_all = oracle.compact(mask, cu)
