@@ -44,13 +44,14 @@ namespace {
 constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int kABytes = BM * BK * 2;               // 16 KB
 constexpr int kBoxBytes = 64 * 64 * 2;             // one 64x64 box of an MN-major operand
-constexpr int kThreads = 192;
+// Threads per CTA: a TMA warp, an MMA warp and four epilogue warps per A sub-tile.
+constexpr int threads_for(int subs) { return 64 + 128 * subs; }
 constexpr int kTmemCols = 512;                     // two 256-column accumulators
 constexpr int kGroupRows = 16;                     // row blocks that share a vocabulary sweep
 constexpr int kTilesPerSplit = 16;                 // vocabulary tiles per work unit
 constexpr int kChunkRows = 8192;                   // rows of the dZ scratch
 constexpr int kMaxPairs = 512;                     // progress marks (one per CTA or CTA pair)
-constexpr int kRowPad = 256;                       // compact rows are padded to a pair's M extent
+constexpr int kRowPad = 512;                       // compact rows are padded to the largest M extent of a work unit
 
 enum Mode { kFwd = 0, kDz = 1, kDh = 2, kDw = 3, kE = 4 };
 
@@ -135,9 +136,9 @@ __device__ __forceinline__ Shape make_shape(const TcParams& p) {
 // Units are ordered so that CTAs running side by side share operands in L2:
 // kFwd/kDz/kE take groups of row blocks (kGroupRows x 128 rows) and, inside a
 // group, walk the vocabulary splits with the row block varying fastest.
-template <int MODE, int CTAS>
+template <int MODE, int CTAS, int SUBS>
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Shape& s, int u) {
-  constexpr int kGroup = kGroupRows / CTAS;
+  constexpr int kGroup = kGroupRows / (CTAS * SUBS);
   Unit w;
   if (MODE == kFwd || MODE == kDz || MODE == kE) {
     const int per_group = kGroup * p.n_splits;
@@ -184,15 +185,18 @@ struct Ring {
   static constexpr int kABytesS = kABytes * SUBS;
   static constexpr int kStage = kABytesS + kBBytes;
   static constexpr int kNum = (192 * 1024) / kStage;
-  static constexpr size_t kSmem = (size_t)kNum * kStage + 1024 /*alignment*/ + 256 /*barriers*/;
+  // SUBS = 2: 4 KB per epilogue warp (32 rows of 128 bytes) from which finished pieces of
+  // the tile leave by TMA store
+  static constexpr int kStaging = SUBS == 2 ? 8 * 4096 : 0;
+  static constexpr size_t kSmem =
+      (size_t)kNum * kStage + kStaging + 1024 /*alignment*/ + 256 /*barriers*/;
 };
 
 template <int MODE, int CTAS, int SUBS>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(threads_for(SUBS), 1)
 nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-              const TcParams p) {
-  static_assert(SUBS == 1 || MODE == kDh || MODE == kDw,
-                "row state that lives across vocabulary tiles needs one sub-tile per thread");
+              const __grid_constant__ CUtensorMap mapC, const TcParams p) {
+  static_assert(SUBS == 1 || CTAS == 2, "two A sub-tiles per CTA are only used by CTA pairs");
   using R = Ring<CTAS, SUBS>;
   constexpr int kNS = R::kNum;
   constexpr int BMU = BM * CTAS * SUBS;
@@ -203,7 +207,8 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kNS * R::kStage);
+  uint8_t* staging = smem + (size_t)kNS * R::kStage;  // 1024-byte aligned like the ring
+  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + R::kStaging);
   uint64_t* full_bar = bars;                   // [kNS]   (CTAS = 2: the even CTA's are used)
   uint64_t* empty_bar = bars + kNS;            // [kNS]
   uint64_t* tfull_bar = bars + 2 * kNS;        // [2]
@@ -224,13 +229,14 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       tc::mbar_init(&tfull_bar[a], 1);
-      tc::mbar_init(&tempty_bar[a], 4 * CTAS);
+      tc::mbar_init(&tempty_bar[a], 4 * SUBS * CTAS);
     }
     *abort_flag = 0u;
     tc::fence_barrier_init();
     tc::fence_proxy_async();
     tc::prefetch_tensormap(&mapA);
     tc::prefetch_tensormap(&mapB);
+    tc::prefetch_tensormap(&mapC);
   }
   if (warp == 1) {
     if (CTAS == 2) {
@@ -255,7 +261,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       uint32_t it = 0;
       bool ok = true;
       for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
-        const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
+        const Unit w = decode_unit<MODE, CTAS, SUBS>(p, shape, u);
         for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt) {
           if ((MODE == kFwd || MODE == kDz || MODE == kE) && rank == 0 && p.progress != nullptr) {
             // Pacing.  The CTAs that sweep the same vocabulary split for different row
@@ -266,7 +272,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             // it is starting and briefly holds back while a mate is more than a tile
             // behind.  Purely advisory: the wait is short and bounded, and results do not
             // depend on it.
-            constexpr int kGroup = kGroupRows / CTAS;
+            constexpr int kGroup = kGroupRows / (CTAS * SUBS);
             volatile unsigned long long* marks = p.progress;
             const int j = nt - w.nt_lo;
             const unsigned long long iter = (unsigned long long)((u - unit0) / unit_stride);
@@ -277,14 +283,21 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
               int mates = shape.mblocks - grp * kGroup;
               mates = mates < kGroup ? mates : kGroup;
               const int first = grp * per_group + w.sp * mates;
-              for (int r = 0; r < mates; ++r) {
-                const int um = first + r;
-                if (um == u) continue;
-                const unsigned long long want = (p.epoch << 40) |
-                                                ((unsigned long long)(um / unit_stride) << 10) |
-                                                (unsigned long long)(j - 1);
-                const int pm = um % unit_stride;
-                for (int spin = 0; spin < 64 && marks[pm] < want; ++spin) __nanosleep(100);
+              // All mates' marks are read together (independent loads, one round trip to
+              // L2), so a pair that is in step with its mates loses well under the time
+              // its shared-memory ring covers.
+              for (int spin = 0; spin < 16; ++spin) {
+                bool behind = false;
+#pragma unroll
+                for (int r = 0; r < kGroup; ++r) {
+                  const int um = first + (r < mates ? r : 0);
+                  const unsigned long long want = (p.epoch << 40) |
+                                                  ((unsigned long long)(um / unit_stride) << 10) |
+                                                  (unsigned long long)(j - 1);
+                  behind |= marks[um % unit_stride] < want;
+                }
+                if (!behind) break;
+                __nanosleep(200);
               }
             }
           }
@@ -306,7 +319,9 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             const int m0 = w.mb * BMU + rank * (BM * SUBS);   // this CTA's rows of A / D
             const int n0 = nt * BN + rank * R::kBRows;        // this CTA's rows of B
             if (MODE == kFwd || MODE == kDz || MODE == kE) {
-              load(a_dst, &mapA, kb * BK, p.row0 + m0);
+#pragma unroll
+              for (int sub = 0; sub < SUBS; ++sub)
+                load(a_dst + sub * kABytes, &mapA, kb * BK, p.row0 + m0 + sub * BM);
               load(b_dst, &mapB, kb * BK, n0);
             } else if (MODE == kDh) {
 #pragma unroll
@@ -350,7 +365,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
-        const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
+        const Unit w = decode_unit<MODE, CTAS, SUBS>(p, shape, u);
         for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt, ++tcount) {
           const uint32_t acc = tcount % kNAcc;
           const uint32_t aph = (tcount / kNAcc) & 1u;
@@ -398,13 +413,14 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------ epilogue (4 warps)
-    const int q = warp & 3;  // tensor-memory lane quadrant this warp may read
+    // ------------------------------------------------ epilogue (4 warps per A sub-tile)
+    const int q = warp & 3;          // tensor-memory lane quadrant this warp may read
+    const int sub = (warp - 2) >> 2;  // the A sub-tile whose rows this warp owns
     const int n_valid = p.row0 + shape.rows;  // compact rows below this are real tokens
     uint32_t tcount = 0;
     bool ok = true;
     for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
-      const Unit w = decode_unit<MODE, CTAS>(p, shape, u);
+      const Unit w = decode_unit<MODE, CTAS, SUBS>(p, shape, u);
       int lrow = 0;  // row inside this launch's M range
       // per-unit row state
       float m_run = -INFINITY, s_run = 0.f, zt_val = 0.f;
@@ -412,7 +428,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       int y = -1;
       float gk = 0.f, lk = 0.f, scale = 1.f;
       bool row_ok = false, over = false;
-      auto load_row = [&](int sub) {  // this thread's row of sub-tile `sub` and its scalars
+      {  // this thread's row and its scalars
         lrow = w.mb * BMU + rank * (BM * SUBS) + sub * BM + q * 32 + lane;
         y = -1;
         gk = 0.f;
@@ -431,8 +447,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         } else {
           row_ok = lrow < p.V;
         }
-      };
-      if (SUBS == 1) load_row(0);
+      }
       for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt, ++tcount) {
         const uint32_t acc = tcount % kNAcc;
         const uint32_t aph = (tcount / kNAcc) & 1u;
@@ -442,11 +457,75 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         if (!ok) break;
         tc::fence_after_sync();
         const int ncols = (MODE == kFwd || MODE == kDz || MODE == kE) ? p.V : p.d;
-#pragma unroll 1
-        for (int sub = 0; sub < SUBS; ++sub) {
-        if (SUBS > 1) load_row(sub);
         const uint32_t taddr =
             tmem_base + ((uint32_t)(q * 32) << 16) + (acc * SUBS + (uint32_t)sub) * BN;
+        if (MODE == kE && SUBS == 2) {
+          // 64 columns at a time: two tensor-memory loads in flight, the numerators of the
+          // warp's 32 rows x 64 columns go to its staging block (128-byte rows in the
+          // 128-byte swizzle) and leave with one TMA store, which writes whole lines.
+          uint8_t* stage = staging + (warp - 2) * 4096;
+          const int row_base = w.mb * BMU + rank * (BM * SUBS) + sub * BM + q * 32;
+          const float nm2 = lk * kLog2e;
+#pragma unroll 1
+          for (int c2 = 0; c2 < BN / 64; ++c2) {
+            const int col0 = nt * BN + c2 * 64;
+            if (col0 >= ncols) break;  // warp-uniform
+            uint32_t ra[32], rb[32];
+            tc::tmem_ld32_issue(taddr + c2 * 64, ra);
+            tc::tmem_ld32_issue(taddr + c2 * 64 + 32, rb);
+            tc::tmem_ld_wait(ra);
+            tc::tmem_ld_pin(rb);
+            const int nv = ncols - col0;  // valid columns from col0 on (may exceed 64)
+            float part = 0.f;
+            uint32_t packed[32];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float e0 = fast_exp2(fmaf(__uint_as_float(ra[2 * j]), kLog2e, -nm2));
+              const float e1 = fast_exp2(fmaf(__uint_as_float(ra[2 * j + 1]), kLog2e, -nm2));
+              if (2 * j < nv) part += e0;
+              if (2 * j + 1 < nv) part += e1;
+              packed[j] = pack_bf16(e0, e1);
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float e0 = fast_exp2(fmaf(__uint_as_float(rb[2 * j]), kLog2e, -nm2));
+              const float e1 = fast_exp2(fmaf(__uint_as_float(rb[2 * j + 1]), kLog2e, -nm2));
+              if (32 + 2 * j < nv) part += e0;
+              if (33 + 2 * j < nv) part += e1;
+              packed[16 + j] = pack_bf16(e0, e1);
+            }
+            if (!row_ok) {  // rows past the last token stay zero
+              part = 0.f;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) packed[j] = 0u;
+            }
+            s_run += part;
+            // Any numerator above e^60 makes the sum exceed it too, so one compare per
+            // piece catches every row that leaves the window.
+            if (part > kWindowSum) over = true;
+            if (y >= col0 && y < col0 + 64) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (col0 + j == y) zt_val = __uint_as_float(ra[j]);
+                if (col0 + 32 + j == y) zt_val = __uint_as_float(rb[j]);
+              }
+              zt_found = true;
+            }
+            // the previous store of this warp has read its staging block
+            if (lane == 0) tc::bulk_wait_read_all();
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<uint4*>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                  make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tc::tma_store_2d(&mapC, stage, col0, row_base);
+              tc::bulk_commit();
+            }
+          }
+        } else
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
           const int col0 = nt * BN + c * 32;
@@ -557,7 +636,6 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             }
           }
         }
-        }  // sub
         tc::fence_before_sync();
         __syncwarp();
         if (lane == 0) {
@@ -580,6 +658,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     }
   }
 
+  if (SUBS == 2 && warp >= 2 && lane == 0) tc::bulk_wait_all();  // this warp's stores are done
   tc::fence_before_sync();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag != 0u) atomicOr(p.status, NAT_DEV_TIMEOUT);
@@ -749,34 +828,42 @@ struct Layout {
       off_hs, off_dz, total;
 };
 
-// Number of vocabulary splits.  Work units of equal length keep the CTAs that sweep the
-// same split in step with each other, which is what lets them share W tiles in L2 (units
-// that differ by a tile drift apart over hundreds of waves and every W tile is then
-// fetched from DRAM several times).  So prefer a divisor of the tile count that gives
-// 8..32 tiles per split, closest to kTilesPerSplit; otherwise fall back to near-equal.
-int pick_splits(int n_tiles) {
-  int best = 0, best_gap = 1 << 30;
+// Number of vocabulary splits.  A work unit of the vocabulary sweeps is (block of rows,
+// split); the CTA pairs take units round-robin, so the sweep of a full row chunk lasts
+// ceil(units / pairs) rounds of about n_tiles / splits tiles each.  Choose the split count
+// that makes this product smallest with 8..32 tiles per unit (long enough to amortise the
+// per-unit state, short enough to balance), preferring lengths near kTilesPerSplit on ties.
+int pick_splits(int n_tiles, int m_units, int slots) {
+  if (slots <= 0) slots = 74;  // CTA pairs of a whole B200; only a tuning assumption
+  if (m_units <= 0) m_units = 1;
+  int best = 0;
+  double best_cost = 0.0;
   for (int s = 1; s <= n_tiles; ++s) {
-    if (n_tiles % s != 0) continue;
-    const int per = n_tiles / s;
-    if (per < 8 || per > 32) continue;
+    const int per = (n_tiles + s - 1) / s;
+    if (per > 32) continue;
+    if (per < 8 && best > 0) break;
+    const long long units = (long long)m_units * s;
+    const long long rounds = (units + slots - 1) / slots;
     const int gap = per > kTilesPerSplit ? per - kTilesPerSplit : kTilesPerSplit - per;
-    if (gap < best_gap) {
-      best_gap = gap;
+    const double cost = (double)rounds * ((double)n_tiles / s) * (1.0 + 1e-4 * gap);
+    if (best == 0 || cost < best_cost) {
       best = s;
+      best_cost = cost;
     }
   }
-  if (best > 0) return best;
-  return (n_tiles + kTilesPerSplit - 1) / kTilesPerSplit;
+  return best > 0 ? best : 1;
 }
+
+int pair_slots();
 
 Layout make_layout(const nat_loss_params& p, int64_t cap) {
   Layout L;
   const int64_t c1 = cap > 0 ? cap : 1;
   L.cap_pad = (int)((c1 + kRowPad - 1) / kRowPad * kRowPad);
   L.n_tiles = (p.V + BN - 1) / BN;
-  L.n_splits = pick_splits(L.n_tiles);
   L.chunk_rows = L.cap_pad < kChunkRows ? L.cap_pad : kChunkRows;
+  // tuned for the single-pass sweep, whose units cover 512 rows on CTA pairs
+  L.n_splits = pick_splits(L.n_tiles, L.chunk_rows / kRowPad, pair_slots());
   L.n_chunks = (L.cap_pad + L.chunk_rows - 1) / L.chunk_rows;
   L.ldz = (p.V + 63) / 64 * 64;
   size_t off = sizeof(WorkspaceHead);
@@ -883,7 +970,7 @@ int pair_slots() {
                              (int)Ring<2, 1>::kSmem) == cudaSuccess) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)sms, 1, 1);
-      cfg.blockDim = dim3(kThreads, 1, 1);
+      cfg.blockDim = dim3(threads_for(1), 1, 1);
       cfg.dynamicSmemBytes = Ring<2, 1>::kSmem;
       cudaLaunchAttribute attr[1];
       attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -913,8 +1000,8 @@ bool g_trace_on = false;
 std::vector<TraceSpan> g_trace_spans;
 
 template <int MODE, int CTAS, int SUBS>
-int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p, int max_units,
-                   cudaStream_t stream) {
+int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
+                   const TcParams& p, int max_units, cudaStream_t stream) {
   static std::atomic<bool> configured[kMaxDevices];
   int dev = 0;
   int sd = current_device(&dev);
@@ -933,7 +1020,7 @@ int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p
   if (groups <= 0) return NAT_OK;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(groups * CTAS), 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.blockDim = dim3(threads_for(SUBS), 1, 1);
   cfg.dynamicSmemBytes = Ring<CTAS, SUBS>::kSmem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -954,7 +1041,7 @@ int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p
     NAT_CUDA(cudaEventCreate(&span.t1));
     NAT_CUDA(cudaEventRecord(span.t0, stream));
   }
-  NAT_CUDA(cudaLaunchKernelEx(&cfg, nat_tc_kernel<MODE, CTAS, SUBS>, a, b, p));
+  NAT_CUDA(cudaLaunchKernelEx(&cfg, nat_tc_kernel<MODE, CTAS, SUBS>, a, b, c, p));
   if (traced) {
     NAT_CUDA(cudaEventRecord(span.t1, stream));
     std::lock_guard<std::mutex> lock(g_trace_mutex);
@@ -967,7 +1054,8 @@ int launch_tc_impl(const CUtensorMap& a, const CUtensorMap& b, const TcParams& p
 // (m_blocks128 * per_block); a pair covers two such blocks per unit.
 template <int MODE>
 int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2,
-              const TcParams& p, int m_blocks128, int per_block, cudaStream_t stream) {
+              const CUtensorMap& c, const TcParams& p, int m_blocks128, int per_block,
+              cudaStream_t stream) {
   // Every launch gets a fresh epoch, so progress marks left by earlier launches (or
   // whatever the workspace held before) compare as "not there yet" or are overwritten
   // by their owner's first tile; either way they cannot stall this launch for long.
@@ -976,12 +1064,12 @@ int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2
   q.epoch = (epoch_counter.fetch_add(1) + 1) & 0x7FFFFFull;
   // The long-K contractions (dH, dW) take two A sub-tiles per CTA; the vocabulary sweeps
   // keep one, because their epilogue state lives across tiles and overlaps the next MMA.
-  constexpr int kSubs = (MODE == kDh || MODE == kDw) ? 2 : 1;
+  constexpr int kSubs = (MODE == kDh || MODE == kDw || MODE == kE) ? 2 : 1;
   if (pair_slots() > 0)
-    return launch_tc_impl<MODE, 2, kSubs>(a, b2, q,
+    return launch_tc_impl<MODE, 2, kSubs>(a, b2, c, q,
                                           ((m_blocks128 + 2 * kSubs - 1) / (2 * kSubs)) * per_block,
                                           stream);
-  return launch_tc_impl<MODE, 1, 1>(a, b1, q, m_blocks128 * per_block, stream);
+  return launch_tc_impl<MODE, 1, 1>(a, b1, c, q, m_blocks128 * per_block, stream);
 }
 
 TokenCtx make_ctx(const LossArgs& a) {
@@ -1073,6 +1161,7 @@ int gather(const LossArgs& a, const Layout& L, const Ws& w) {
 
 struct Maps {
   CUtensorMap hcK, wK, wK2, dzK, wMn, dzMn, hcMn, hsMn;  // wK2: 128-row boxes for CTA pairs
+  CUtensorMap dzSt;  // the numerator scratch as a store target: 64 columns x 32 rows
 };
 
 int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
@@ -1086,6 +1175,7 @@ int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
   if ((s = make_map(&m->dzMn, w.dz, a.p.V, L.chunk_rows, zpitch, 64, BK)) != NAT_OK) return s;
   if ((s = make_map(&m->hcMn, w.hc, a.p.d, L.cap_pad, dpitch, 64, BK)) != NAT_OK) return s;
   if ((s = make_map(&m->hsMn, w.hs, a.p.d, L.chunk_rows, dpitch, 64, BK)) != NAT_OK) return s;
+  if ((s = make_map(&m->dzSt, w.dz, a.p.V, L.chunk_rows, zpitch, 64, 32)) != NAT_OK) return s;
   return NAT_OK;
 }
 
@@ -1107,9 +1197,9 @@ int launch_two_pass_chunk(const LossArgs& a, const Layout& L, const Ws& w, const
   p.run_if = 1;
   const int mb = L.chunk_rows / BM;
   const int nb_d = (a.p.d + BN - 1) / BN;
-  if ((s = launch_tc<kDz>(m.hcK, m.wK, m.wK2, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
-  if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, p, mb, nb_d, a.stream)) != NAT_OK) return s;
-  return launch_tc<kDw>(m.dzMn, m.hcMn, m.hcMn, p, (a.p.V + BM - 1) / BM, nb_d, a.stream);
+  if ((s = launch_tc<kDz>(m.hcK, m.wK, m.wK2, m.hcK, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
+  if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, m.hcK, p, mb, nb_d, a.stream)) != NAT_OK) return s;
+  return launch_tc<kDw>(m.dzMn, m.hcMn, m.hcMn, m.hcK, p, (a.p.V + BM - 1) / BM, nb_d, a.stream);
 }
 
 int launch_onehot(const LossArgs& a, const Ws& w) {
@@ -1138,7 +1228,7 @@ int loss_bf16_fwd(const LossArgs& a) {
     Maps m;
     if ((s = make_maps(a, L, w, &m)) != NAT_OK) return s;
     const TcParams p = base_params(a, L, w);
-    if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, p, L.cap_pad / BM, L.n_splits, a.stream)) !=
+    if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, m.hcK, p, L.cap_pad / BM, L.n_splits, a.stream)) !=
         NAT_OK)
       return s;
     fwd_finalize_kernel<<<finalize_grid((int)a.cap), 256, 0, a.stream>>>(
@@ -1192,7 +1282,7 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.V = a.p.V < BN ? a.p.V : BN;
       p.n_splits = 1;
       p.part_m = w.mref;
-      if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, p, L.cap_pad / BM, 1, a.stream)) != NAT_OK)
+      if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, m.hcK, p, L.cap_pad / BM, 1, a.stream)) != NAT_OK)
         return s;
     }
     for (int ci = 0; ci < L.n_chunks; ++ci) {
@@ -1202,7 +1292,7 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.row0 = row0;
       p.chunk_rows = L.chunk_rows;
       p.ovf = ovf;
-      if ((s = launch_tc<kE>(m.hcK, m.wK, m.wK2, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
+      if ((s = launch_tc<kE>(m.hcK, m.wK, m.wK2, m.dzSt, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
       fused_finalize_kernel<<<L.chunk_rows < 2048 ? L.chunk_rows : 2048, 128, 0, a.stream>>>(
           c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_splits, L.cap_pad, w.mref, w.ps, w.zt,
           a.dloss, a.logp, a.lse, w.term, w.g, w.cs, w.hc, w.hs, a.p.d, ovf);
@@ -1212,8 +1302,8 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.run_if = 0;
       p.row_scale = w.cs;
       p.b_row0 = 0;  // Hs is local to the chunk
-      if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, p, mb, nb_d, a.stream)) != NAT_OK) return s;
-      if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, m.hsMn, p, (a.p.V + BM - 1) / BM, nb_d,
+      if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, m.hcK, p, mb, nb_d, a.stream)) != NAT_OK) return s;
+      if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, m.hsMn, m.hcK, p, (a.p.V + BM - 1) / BM, nb_d,
                               a.stream)) != NAT_OK)
         return s;
       // Predicated redo of the chunk by the two-pass kernels (no-ops unless *ovf != 0).
@@ -1222,7 +1312,7 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       pf.chunk_rows = L.chunk_rows;
       pf.flag = ovf;
       pf.run_if = 1;
-      if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, pf, mb, L.n_splits, a.stream)) != NAT_OK)
+      if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, m.hcK, pf, mb, L.n_splits, a.stream)) != NAT_OK)
         return s;
       fwd_finalize_kernel<<<finalize_grid(L.chunk_rows), 256, 0, a.stream>>>(
           c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_splits, L.cap_pad, w.pm, w.ps, w.zt,
