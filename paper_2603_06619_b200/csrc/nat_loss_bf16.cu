@@ -186,7 +186,7 @@ struct Ring {
   static constexpr int kStage = kABytesS + kBBytes;
   static constexpr int kNum = (192 * 1024) / kStage;
   // SUBS = 2: 4 KB per epilogue warp (32 rows of 128 bytes) from which finished pieces of
-  // the tile leave by TMA store
+  // the tile leave by TMA store (kE) or TMA reduction (kDw)
   static constexpr int kStaging = SUBS == 2 ? 8 * 4096 : 0;
   static constexpr size_t kSmem =
       (size_t)kNum * kStage + kStaging + 1024 /*alignment*/ + 256 /*barriers*/;
@@ -623,6 +623,25 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 dst[g8] = make_uint4(o[0], o[1], o[2], o[3]);
               }
             }
+          } else if (SUBS == 2) {
+            // dW += tile: the warp's 32 rows x 32 columns go to its staging block (128-byte
+            // rows in the 128-byte swizzle) and leave as one TMA reduction, which the L2
+            // applies to whole lines; rows past V are clipped by the tensor map.  Every
+            // element is touched once per launch and launches are stream-ordered, so the
+            // sum's order is fixed.
+            uint8_t* stage = staging + (warp - 2) * 4096;
+            if (lane == 0) tc::bulk_wait_read_all();  // the previous reduction has read the block
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<float4*>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                  make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tc::tma_reduce_add_2d(&mapC, stage, col0, lrow);
+              tc::bulk_commit();
+            }
           } else {
             if (row_ok) {
               // dW += tile: 16-byte reductions performed by the L2 (nothing comes back to
@@ -928,6 +947,24 @@ int make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows,
   return NAT_OK;
 }
 
+// float32 matrix [rows, inner] as a reduction target: box = 32 x 32 elements (128-byte rows).
+int make_map_f32(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows) {
+  EncodeTiledFn enc;
+  int s = get_encoder(&enc);
+  if (s != NAT_OK) return s;
+  const cuuint64_t dims[2] = {inner, rows};
+  const cuuint64_t strides[1] = {inner * 4};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims,
+                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(NAT_ERR_CUDA, "cuTensorMapEncodeTiled (float32) failed with code %d", (int)r);
+  return NAT_OK;
+}
+
 // Per-device facts are cached per device index: one process may drive several GPUs.
 constexpr int kMaxDevices = 64;
 
@@ -1162,6 +1199,7 @@ int gather(const LossArgs& a, const Layout& L, const Ws& w) {
 struct Maps {
   CUtensorMap hcK, wK, wK2, dzK, wMn, dzMn, hcMn, hsMn;  // wK2: 128-row boxes for CTA pairs
   CUtensorMap dzSt;  // the numerator scratch as a store target: 64 columns x 32 rows
+  CUtensorMap dwRed;  // dW as a reduction target (valid only when the call has a dW)
 };
 
 int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
@@ -1176,6 +1214,8 @@ int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
   if ((s = make_map(&m->hcMn, w.hc, a.p.d, L.cap_pad, dpitch, 64, BK)) != NAT_OK) return s;
   if ((s = make_map(&m->hsMn, w.hs, a.p.d, L.chunk_rows, dpitch, 64, BK)) != NAT_OK) return s;
   if ((s = make_map(&m->dzSt, w.dz, a.p.V, L.chunk_rows, zpitch, 64, 32)) != NAT_OK) return s;
+  m->dwRed = m->dzSt;
+  if (a.dW != nullptr && (s = make_map_f32(&m->dwRed, a.dW, a.p.d, a.p.V)) != NAT_OK) return s;
   return NAT_OK;
 }
 
@@ -1199,7 +1239,7 @@ int launch_two_pass_chunk(const LossArgs& a, const Layout& L, const Ws& w, const
   const int nb_d = (a.p.d + BN - 1) / BN;
   if ((s = launch_tc<kDz>(m.hcK, m.wK, m.wK2, m.hcK, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
   if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, m.hcK, p, mb, nb_d, a.stream)) != NAT_OK) return s;
-  return launch_tc<kDw>(m.dzMn, m.hcMn, m.hcMn, m.hcK, p, (a.p.V + BM - 1) / BM, nb_d, a.stream);
+  return launch_tc<kDw>(m.dzMn, m.hcMn, m.hcMn, m.dwRed, p, (a.p.V + BM - 1) / BM, nb_d, a.stream);
 }
 
 int launch_onehot(const LossArgs& a, const Ws& w) {
@@ -1303,7 +1343,7 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.row_scale = w.cs;
       p.b_row0 = 0;  // Hs is local to the chunk
       if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, m.hcK, p, mb, nb_d, a.stream)) != NAT_OK) return s;
-      if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, m.hsMn, m.hcK, p, (a.p.V + BM - 1) / BM, nb_d,
+      if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, m.hsMn, m.dwRed, p, (a.p.V + BM - 1) / BM, nb_d,
                               a.stream)) != NAT_OK)
         return s;
       // Predicated redo of the chunk by the two-pass kernels (no-ops unless *ovf != 0).
