@@ -47,7 +47,7 @@ constexpr int kBoxBytes = 64 * 64 * 2;             // one 64x64 box of an MN-maj
 // Threads per CTA: a TMA warp, an MMA warp and four epilogue warps per A sub-tile.
 constexpr int threads_for(int subs) { return 64 + 128 * subs; }
 constexpr int kTmemCols = 512;                     // two 256-column accumulators
-constexpr int kGroupRows = 16;                     // row blocks that share a vocabulary sweep
+constexpr int kGroupRows = 32;                     // row blocks that share a vocabulary sweep
 constexpr int kTilesPerSplit = 16;                 // vocabulary tiles per work unit
 constexpr int kChunkRows = 8192;                   // rows of the dZ scratch
 constexpr int kMaxPairs = 512;                     // progress marks (one per CTA or CTA pair)
