@@ -355,7 +355,7 @@ def run_ours(args, w):
         # DRAM bytes per launch (one 8192-row chunk of this head) from the ncu capture
         # summarised in profiles/nat_tc_kernel_qwen3_8b_chunk.md; null for other shapes
         if w.name == "qwen3_8b":
-            traffic = {"e": 9.13e9, "dh": 10.83e9, "dw": 20.0e9}.get(top)
+            traffic = {"e": 9.51e9, "dh": 16.79e9, "dw": 21.37e9}.get(top)
     call_tflops = roof_flops / (roof_ms * 1e-3) / 1e12
 
     line = {
@@ -419,8 +419,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen3_8b")
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--ref-rows", type=int, default=128,
-                    help="selected rows the fp64 oracle evaluates per timed sample (about 12 s on 16 cores)")
+    ap.add_argument("--ref-rows", type=int, default=384,
+                    help="selected rows the fp64 oracle evaluates per timed sample (about 15 s on 16 cores)")
     ap.add_argument("--allreduce-dw", action="store_true",
                     help="N > 1: sum loss and dW over the ranks inside every step (the exchange of "
                          "a data-parallel trainer); off by default: ranks then run independent "

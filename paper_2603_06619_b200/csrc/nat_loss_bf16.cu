@@ -9,7 +9,7 @@
 //   kDz   S = Hc W^T  recomputed         epilogue: -g exp(S - lse) -> bf16 into
 //                                        the bounded scratch dZ[chunk, V].
 //   kDh   dH = dZ W   (rows x d, K = V)  epilogue: + g W[y] (one-hot term) -> bf16.
-//   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 reduction into dW (red.global.add).
+//   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 reduction into dW (TMA reduce-add).
 //   kE    S = Hc W^T  single-pass variant  epilogue: E = exp(S - mref) -> bf16 into the
 //                                        same scratch, row sums of E, target pick.
 //
@@ -23,9 +23,13 @@
 // row's reference by more than 60 (E would leave the fp32/bf16 range) is redone by the
 // two-pass kernels, which are launched predicated on the chunk's flag.
 //
-// Roles per CTA (192 threads): warp 0 issues TMA loads into a 4-stage shared
-// memory ring, warp 1 issues tcgen05.mma into one of two 128x256 fp32
-// accumulators in tensor memory, warps 2..5 drain the other accumulator.
+// Roles per CTA: warp 0 issues TMA loads into a shared-memory ring, warp 1 issues
+// tcgen05.mma into fp32 accumulators in tensor memory, four epilogue warps per A sub-tile
+// drain them.  kFwd / kDz: one sub-tile, two 128x256 accumulators, so one tile's epilogue
+// overlaps the next tile's MMAs.  kE / kDh / kDw: two sub-tiles per CTA (512x256 per CTA
+// pair, a quarter less operand traffic); their accumulators fill tensor memory, the
+// epilogue is exposed and therefore leaves through a shared-memory staging block by TMA
+// store (kE) or TMA reduction (kDw) instead of scattered 16-byte accesses.
 // Every mbarrier wait is bounded; a wait that runs out raises the block's
 // abort flag and NAT_DEV_TIMEOUT in the workspace's status word.
 #include <cuda_bf16.h>
