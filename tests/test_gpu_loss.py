@@ -185,6 +185,45 @@ def test_fused_accumulate_and_dloss():
     assert parity.rel_fro(st.dH[:n].float().cpu().numpy(), -2 * baseH[:n].float().cpu().numpy()) < 1e-2
 
 
+def test_fused_compact_hidden_layout():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=4, device="cuda")
+    nb = wl.to_numpy(batch)
+    ref_sel = parity.oracle_selection(w, nb, 4, 0)
+    idx = torch.from_numpy(ref_sel["sel_idx"]).long().cuda()
+    compact = dict(batch, hidden=batch["hidden"][idx].contiguous())
+    st = parity.gpu_step(w, compact, 4, 0, hidden_is_compact=True, fused=True)
+    parity.check_selection(st, ref_sel, w)
+    parity.check_loss(st, ref_sel, nb, w)
+
+
+def test_fused_empty_selection_capacity_and_reruns():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    args = (batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], batch["cu_seqlens"])
+    st = parity.gpu_step(w, batch, 0, 0, fused=True)
+    loss1, logp1, dH1 = st.loss.clone(), st.logp.clone(), st.dH.clone()
+    st.run(batch, w.sel_mode, p=w.p, seed=0, fused=True)
+    torch.cuda.synchronize()
+    n = int(st.n_sel.item())
+    assert torch.equal(loss1, st.loss) and torch.equal(logp1[:n], st.logp[:n])
+    assert torch.equal(dH1[:n], st.dH[:n])            # dense parts are order-fixed
+    # nothing selected: loss 0 and zero dW
+    st.mask.zero_()
+    st.compact(batch["cu_seqlens"])
+    st.loss_fwd_bwd(*args)
+    torch.cuda.synchronize()
+    assert int(st.n_sel.item()) == 0 and float(st.loss.item()) == 0.0
+    assert float(st.dW.abs().max().item()) == 0.0 and st.status() == 0
+    # more tokens selected than the stated capacity: reported, the first rows are still right
+    cap = 300                                          # not a multiple of any tile extent
+    st2 = parity.gpu_step(w, batch, 0, 0, fused=True, n_sel_cap=cap)
+    assert int(st2.n_sel.item()) > cap
+    assert st2.status() & nat.NAT_DEV_CAPACITY
+    assert float((st2.logp[:cap] - logp1[:cap]).abs().max()) < parity.TOL_LOGP
+    assert parity.rel_fro(st2.dH[:cap].float().cpu().numpy(), dH1[:cap].float().cpu().numpy()) < 1e-2
+
+
 def test_trace_reports_per_kernel_time():
     w = wl.WORKLOADS["mid"]
     batch = wl.make_batch(w, seed=0, device="cuda")
