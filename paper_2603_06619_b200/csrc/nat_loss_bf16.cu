@@ -837,10 +837,15 @@ __global__ void onehot_dw_kernel(const __nv_bfloat16* __restrict__ Hc,
     const float gk = g[k];
     if (gk == 0.f) continue;
     const int y = targets[sel_idx[k]];
-    const __nv_bfloat16* h = Hc + (size_t)k * d;
+    const uint2* h = reinterpret_cast<const uint2*>(Hc + (size_t)k * d);  // four bf16 at a time
     float* dst = dW + (size_t)y * d;
-    for (int j = threadIdx.x; j < d; j += blockDim.x)
-      atomicAdd(dst + j, gk * __bfloat162float(h[j]));
+    for (int j = threadIdx.x; j < d / 4; j += blockDim.x) {
+      const uint2 hv = h[j];
+      const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&hv.x);
+      const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&hv.y);
+      tc::red_add_f32x4(dst + 4 * j, gk * __low2float(lo), gk * __high2float(lo),
+                        gk * __low2float(hi), gk * __high2float(hi));
+    }
   }
 }
 
