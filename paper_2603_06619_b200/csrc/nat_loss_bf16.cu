@@ -189,9 +189,9 @@ struct Ring {
   static constexpr int kABytesS = kABytes * SUBS;
   static constexpr int kStage = kABytesS + kBBytes;
   static constexpr int kNum = (192 * 1024) / kStage;
-  // SUBS = 2: 4 KB per epilogue warp (32 rows of 128 bytes) from which finished pieces of
+  // CTA pairs: 4 KB per epilogue warp (32 rows of 128 bytes) from which finished pieces of
   // the tile leave by TMA store (kE) or TMA reduction (kDw)
-  static constexpr int kStaging = SUBS == 2 ? 8 * 4096 : 0;
+  static constexpr int kStaging = CTAS == 2 ? 4 * SUBS * 4096 : 0;
   static constexpr size_t kSmem =
       (size_t)kNum * kStage + kStaging + 1024 /*alignment*/ + 256 /*barriers*/;
 };
@@ -463,7 +463,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         const int ncols = (MODE == kFwd || MODE == kDz || MODE == kE) ? p.V : p.d;
         const uint32_t taddr =
             tmem_base + ((uint32_t)(q * 32) << 16) + (acc * SUBS + (uint32_t)sub) * BN;
-        if (MODE == kE && SUBS == 2) {
+        if (MODE == kE && CTAS == 2) {
           // 64 columns at a time: two tensor-memory loads in flight, the numerators of the
           // warp's 32 rows x 64 columns go to its staging block (128-byte rows in the
           // 128-byte swizzle) and leave with one TMA store, which writes whole lines.
@@ -681,7 +681,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
     }
   }
 
-  if (SUBS == 2 && warp >= 2 && lane == 0) tc::bulk_wait_all();  // this warp's stores are done
+  if (CTAS == 2 && warp >= 2 && lane == 0) tc::bulk_wait_all();  // this warp's stores are done
   tc::fence_before_sync();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag != 0u) atomicOr(p.status, NAT_DEV_TIMEOUT);
@@ -884,14 +884,17 @@ int pick_splits(int n_tiles, int m_units, int slots) {
 
 int pair_slots();
 
+// Hidden sizes from which the single-pass sweep uses 512-row work units (see launch_tc).
+bool wide_sweep(int d) { return d >= 2048; }
+
 Layout make_layout(const nat_loss_params& p, int64_t cap) {
   Layout L;
   const int64_t c1 = cap > 0 ? cap : 1;
   L.cap_pad = (int)((c1 + kRowPad - 1) / kRowPad * kRowPad);
   L.n_tiles = (p.V + BN - 1) / BN;
   L.chunk_rows = L.cap_pad < kChunkRows ? L.cap_pad : kChunkRows;
-  // tuned for the single-pass sweep, whose units cover 512 rows on CTA pairs
-  L.n_splits = pick_splits(L.n_tiles, L.chunk_rows / kRowPad, pair_slots());
+  // tuned for the single-pass sweep, whose units cover 512 or 256 rows on CTA pairs
+  L.n_splits = pick_splits(L.n_tiles, L.chunk_rows / (wide_sweep(p.d) ? 512 : 256), pair_slots());
   L.n_chunks = (L.cap_pad + L.chunk_rows - 1) / L.chunk_rows;
   L.ldz = (p.V + 63) / 64 * 64;
   size_t off = sizeof(WorkspaceHead);
@@ -1108,13 +1111,18 @@ int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2
   static std::atomic<unsigned long long> epoch_counter{0};
   TcParams q = p;
   q.epoch = (epoch_counter.fetch_add(1) + 1) & 0x7FFFFFull;
-  // The long-K contractions (dH, dW) take two A sub-tiles per CTA; the vocabulary sweeps
-  // keep one, because their epilogue state lives across tiles and overlaps the next MMA.
-  constexpr int kSubs = (MODE == kDh || MODE == kDw || MODE == kE) ? 2 : 1;
-  if (pair_slots() > 0)
-    return launch_tc_impl<MODE, 2, kSubs>(a, b2, c, q,
-                                          ((m_blocks128 + 2 * kSubs - 1) / (2 * kSubs)) * per_block,
-                                          stream);
+  // dH and dW (long K) always take two A sub-tiles per CTA.  The single-pass sweep kE takes
+  // two when the hidden size is large: its 512x256 tile fills tensor memory, so its epilogue
+  // is exposed, which pays only while a tile's MMAs (proportional to d) dwarf it; for small d
+  // it keeps 256x256 tiles whose epilogue overlaps the next tile.  kFwd / kDz keep one.
+  if (pair_slots() > 0) {
+    const bool two = MODE == kDh || MODE == kDw || (MODE == kE && wide_sweep(p.d));
+    if (two)
+      return launch_tc_impl<MODE, 2, (MODE == kFwd || MODE == kDz) ? 1 : 2>(
+          a, b2, c, q, ((m_blocks128 + 3) / 4) * per_block, stream);
+    return launch_tc_impl<MODE, 2, (MODE == kDh || MODE == kDw) ? 2 : 1>(
+        a, b2, c, q, ((m_blocks128 + 1) / 2) * per_block, stream);
+  }
   return launch_tc_impl<MODE, 1, 1>(a, b1, c, q, m_blocks128 * per_block, stream);
 }
 
