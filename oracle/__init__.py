@@ -18,6 +18,12 @@ Parity status of each function (what pins it to something other than itself):
                     ceil(p 2^24), the uniform-cutoff schedule reproducing the uniform law,
                     prefix structure, and exhaustive enumeration of a geometric cut law
                     showing the HT estimator unbiased (Proposition 1).
+  select_cutlaw     pinned: the three properties of Eq. rpc-survival (pi_1 = 1, monotone,
+                    positive where the law has mass), pi against the suffix sums of q in
+                    rational arithmetic, the uniform law reproducing the uniform-cutoff
+                    closed form bit for bit, draw boundaries against the exact integer
+                    count, cut frequencies over seeds, and exhaustive enumeration of the
+                    cuts showing the HT estimator unbiased (Proposition 1).
   compact           pinned: brute-force list comprehension, segment structure
                     for prefix modes.
   gather/scatter    pinned: numpy fancy indexing, scatter(gather(x)) = mask * x, and the
@@ -29,6 +35,8 @@ Parity status of each function (what pins it to something other than itself):
   policy_loss_bwd   pinned: central finite differences of policy_loss_fwd,
                     zero column sums, exhaustive enumeration of the gradient's
                     expectation, saturated-clip zero gradient.
+  policy_loss_dW_rows  pinned: equals the corresponding rows of policy_loss_bwd's dW (itself
+                    pinned by finite differences) and central differences on the chosen rows.
 """
 from .philox import philox4x32_10  # noqa: F401
 from .nat_oracle import (  # noqa: F401
@@ -38,9 +46,13 @@ from .nat_oracle import (  # noqa: F401
     grpo_adv,
     select,
     select_survival,
+    select_cutlaw,
+    cutlaw_counts,
     compact,
     gather_rows,
     scatter_rows,
     policy_loss_fwd,
     policy_loss_bwd,
+    policy_loss_dW_rows,
+    grad_coeff,
 )

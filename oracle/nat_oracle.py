@@ -79,10 +79,15 @@ def urs_threshold(p):
     return min(max(thr, 1), 1 << 32)
 
 
-def select(mode, cu_seqlens, *, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
+def select(mode, cu_seqlens, *, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0, resp_base=0):
     """Draw the mask m, the inclusion probabilities pi and the per-response cut.
 
     Returns (mask uint8 [N_tot], pi float32 [N_tot], cut_len int32 [B] or None).
+
+    ``resp_base`` is the index, in the whole job's batch, of the first response of
+    ``cu_seqlens``: the draws of local response i are those of response resp_base + i, so a
+    shard of a batch realises the same mask as the whole batch does for those responses
+    (masks of different responses are independent, Section 3.1).
 
     URS: token t of response i consumes word (t-1) mod 4 of the Philox block
     with counter ((t-1) div 4, i, 0, offset_lo); m = [x < thr], pi = thr/2^32.
@@ -109,7 +114,7 @@ def select(mode, cu_seqlens, *, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
             if T == 0:
                 continue
             t0 = np.arange(T, dtype=np.uint64)          # t - 1
-            words = philox4x32_10(t0 >> np.uint64(2), i, 0, off_lo, k0, k1)
+            words = philox4x32_10(t0 >> np.uint64(2), resp_base + i, 0, off_lo, k0, k1)
             x = np.choose((t0 & np.uint64(3)).astype(np.int64), words)
             mask[cu[i]:cu[i + 1]] = (x < np.uint64(thr)).astype(np.uint8)
             pi[cu[i]:cu[i + 1]] = pi_val
@@ -123,7 +128,7 @@ def select(mode, cu_seqlens, *, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
         if mode == SEL_RPC:
             C = min(max(int(min_cut), 1), T)
             n = T - C + 1
-            x0, x1, _, _ = philox4x32_10(0, i, 1, off_lo, k0, k1)
+            x0, x1, _, _ = philox4x32_10(0, resp_base + i, 1, off_lo, k0, k1)
             u = (int(x1) << 32) | int(x0)
             L = C + ((u * n) >> 64)
             num = (T - t + 1).astype(np.float32)
@@ -142,7 +147,7 @@ def select(mode, cu_seqlens, *, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
     return mask, pi, cut_len
 
 
-def select_survival(cu_seqlens, surv, *, seed=0, offset=0):
+def select_survival(cu_seqlens, surv, *, seed=0, offset=0, resp_base=0):
     """Random Prefix Cutting under a caller-given survival schedule (Eq. rpc-mask,
     Eq. rpc-survival with a general cut law q_i).
 
@@ -151,7 +156,7 @@ def select_survival(cu_seqlens, surv, *, seed=0, offset=0):
     u = (x0 >> 8) * 2^-24 from the Philox block with counter (0, i, 2, offset_lo); then
     L_i >= t  <=>  u < p_{i,t}, so m_t = [u < surv[n]] (a prefix because surv is monotone)
     and Pr(L_i >= t) = ceil(p_{i,t} 2^24) / 2^24, within 2^-24 of the schedule.
-    The inclusion probabilities are the schedule itself.
+    The inclusion probabilities are the schedule itself.  ``resp_base`` as in ``select``.
 
     Returns (mask uint8 [N_tot], cut_len int32 [B]).
     """
@@ -168,12 +173,75 @@ def select_survival(cu_seqlens, surv, *, seed=0, offset=0):
         p = surv[lo:hi]
         if p[0] != 1.0 or np.any(np.diff(p) > 0) or p[-1] <= 0:
             raise ValueError("survival schedule must start at 1, not increase and stay positive")
-        x0, _, _, _ = philox4x32_10(0, i, 2, off_lo, k0, k1)
+        x0, _, _, _ = philox4x32_10(0, resp_base + i, 2, off_lo, k0, k1)
         u = np.float32(int(x0) >> 8) * np.float32(2.0 ** -24)
         m = u < p
         mask[lo:hi] = m.astype(np.uint8)
         cut_len[i] = int(m.sum())
     return mask, cut_len
+
+
+def cutlaw_counts(q):
+    """Cut-law masses in 32-bit fixed point: k = floor(min(q, 1) * 2^32) for q > 0, else 0.
+
+    The scaling by a power of two and the floor are exact, so the counts (and every sum of
+    them, taken in 64-bit integers) do not depend on the order of evaluation.
+    """
+    q = np.asarray(q, dtype=np.float32)
+    k = np.zeros(q.shape, dtype=np.uint64)
+    pos = q > 0                                     # NaN and negative masses count as zero
+    scaled = np.minimum(q[pos], np.float32(1.0)).astype(np.float64) * 4294967296.0
+    k[pos] = np.floor(scaled).astype(np.uint64)
+    return k
+
+
+def select_cutlaw(cu_seqlens, q, *, seed=0, offset=0, resp_base=0):
+    """Random Prefix Cutting under a caller-given cut law q_i (Eq. rpc-mask, Eq. rpc-survival).
+
+    ``q[n]`` is the (unnormalised) mass the cut law of token n's response puts on cutting
+    right after that token, q_i(l) up to a common factor per response.  With the fixed-point
+    counts k of ``cutlaw_counts``:
+        S_t  = sum_{l >= t} k_l                 (Eq. rpc-survival's suffix sum, exact integers)
+        pi_t = float32(double(S_t) / double(S_1))      so pi_1 = 1, pi non-increasing
+        u    = x1 2^32 + x0 from the Philox block with counter (0, resp_base + i, 3, offset_lo)
+        r    = floor(u S_1 / 2^64)              uniform on {0 .. S_1 - 1} to within S_1 2^-64
+        m_t  = [S_t > r]                        i.e. L_i = max{t : S_t > r}, Pr(L_i >= t) = S_t / S_1
+    A response whose counts are all zero is kept whole with pi = 1.
+
+    Returns (mask uint8 [N_tot], pi float32 [N_tot], cut_len int32 [B]).
+    """
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    B = cu.shape[0] - 1
+    n_tot = int(cu[B])
+    k = cutlaw_counts(q)
+    assert k.shape == (n_tot,)
+    mask = np.zeros(n_tot, dtype=np.uint8)
+    pi = np.zeros(n_tot, dtype=np.float32)
+    cut_len = np.zeros(B, dtype=np.int32)
+    k0, k1, off_lo = _key(seed, offset)
+    for i in range(B):
+        lo, hi = int(cu[i]), int(cu[i + 1])
+        if hi == lo:
+            continue
+        S = [0] * (hi - lo)                         # Python integers: exact
+        run = 0
+        for t in range(hi - lo - 1, -1, -1):
+            run += int(k[lo + t])
+            S[t] = run
+        total = S[0]
+        if total == 0:
+            mask[lo:hi] = 1
+            pi[lo:hi] = np.float32(1.0)
+            cut_len[i] = hi - lo
+            continue
+        x0, x1, _, _ = philox4x32_10(0, resp_base + i, 3, off_lo, k0, k1)
+        u = (int(x1) << 32) | int(x0)
+        r = (u * total) >> 64
+        S64 = np.array(S, dtype=np.uint64)
+        mask[lo:hi] = (S64 > np.uint64(r)).astype(np.uint8)
+        pi[lo:hi] = (S64.astype(np.float64) / np.float64(np.uint64(total))).astype(np.float32)
+        cut_len[i] = int(mask[lo:hi].sum())
+    return mask, pi, cut_len
 
 
 # --------------------------------------------------------------------------
@@ -356,3 +424,40 @@ def policy_loss_bwd(hidden, W, targets, old_logp, adv, pi, cu_seqlens, sel_idx, 
     out = dict(fwd)
     out.update(dH=dH, dW=dW, g=g, dH_dense=dH_dense, dW_dense=dW_dense)
     return out
+
+
+def policy_loss_dW_rows(hidden_blocks, W_rows, v_ids, y, g, lse):
+    """Rows ``v_ids`` of dW, summed over ALL selected tokens, from per-token scalars.
+
+        dW[v, :] = sum_n g_n (1[v = y_n] - exp(W_v . h_n - lse_n)) h_n
+
+    which is ``policy_loss_bwd``'s dW restricted to a few vocabulary rows: the softmax
+    probability of entry v needs only W_v, h_n and the row's lse_n.  ``hidden_blocks``
+    yields the selected rows in order as consecutive arrays [rows, d] (so a caller can
+    stream them), ``W_rows`` is W[v_ids] (float [len(v_ids), d]), ``y`` the selected tokens'
+    targets, ``g`` their gradient coefficients (``grad_coeff``) and ``lse`` their
+    log-sum-exp, all [n_sel].
+
+    Returns (dW_rows, dW_rows_dense) float64 [len(v_ids), d]; the second leaves out the
+    one-hot target term.
+    """
+    Wv = np.asarray(W_rows, dtype=np.float64)
+    v_ids = np.asarray(v_ids, dtype=np.int64)
+    y = np.asarray(y, dtype=np.int64)
+    g = np.asarray(g, dtype=np.float64)
+    lse = np.asarray(lse, dtype=np.float64)
+    out = np.zeros(Wv.shape)
+    dense = np.zeros(Wv.shape)
+    lo = 0
+    for blk in hidden_blocks:
+        h = np.asarray(blk, dtype=np.float64)
+        hi = lo + h.shape[0]
+        z = h @ Wv.T                                         # [rows, len(v_ids)]
+        dz_dense = -g[lo:hi, None] * np.exp(z - lse[lo:hi, None])
+        hit = (y[lo:hi, None] == v_ids[None, :])
+        dz = dz_dense + np.where(hit, g[lo:hi, None], 0.0)
+        out += dz.T @ h
+        dense += dz_dense.T @ h
+        lo = hi
+    assert lo == y.shape[0]
+    return out, dense

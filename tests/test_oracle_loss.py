@@ -11,8 +11,8 @@ import numpy as np
 import pytest
 from scipy.special import log_softmax
 
-from oracle import (SEL_DET, SEL_RPC, SEL_URS, compact, grpo_adv, policy_loss_bwd,
-                    policy_loss_fwd, select)
+from oracle import (SEL_DET, SEL_RPC, SEL_URS, compact, grad_coeff, grpo_adv, policy_loss_bwd,
+                    policy_loss_dW_rows, policy_loss_fwd, select, select_cutlaw)
 from paper_2603_06619_b200 import workloads as wl
 
 
@@ -279,11 +279,19 @@ def test_rpc_enumeration_is_unbiased_and_det_is_biased():
             np.testing.assert_allclose(e_dW, full["dW"], atol=2e-7 * scale)
             full_dH = _scatter_dH(full, np.nonzero(only)[0], b["n_tot"], w.d)
             np.testing.assert_allclose(e_dH, full_dH, atol=2e-7 * np.abs(full_dH).max())
-            # variance in stopping-time form (Appendix B.1):
-            # Var = E[(sum_{t<=tau} L_t/p_t)^2]/T^2 - (sum_t L_t)^2/T^2
+            # Variance in stopping-time form (Eq. rpc-variance-stopping, Appendix B.1),
+            # evaluated from the per-token losses L_t of the full-token run and the
+            # survival probabilities, not from the estimator's own realisations:
+            #   Var[mu_hat] = (E[(sum_{t<=tau} L_t/p_t)^2] - (sum_t L_t)^2) / T^2,
+            # tau uniform on {C..T}.  The loss of a batch whose mask covers response i
+            # only is -mu_hat_i / B.
+            Lt = full["L"]                                     # per-token losses, t = 1..T
+            pt = pi[cu[i]:cu[i + 1]].astype(np.float64)
+            partial = np.cumsum(Lt / pt)                       # sum_{t<=tau} L_t / p_t
+            second = np.mean(partial[Ci - 1:] ** 2)            # E over tau = C..T
+            var_formula = (second - Lt.sum() ** 2) / T ** 2 / w.B ** 2
             var_direct = np.mean((np.array(losses) - np.mean(losses)) ** 2)
-            var_formula = np.mean(np.array(losses) ** 2) - full["loss"] ** 2
-            assert abs(var_direct - var_formula) < 1e-6 * (abs(var_formula) + 1e-9) + 1e-12
+            assert abs(var_direct - var_formula) < 2e-6 * abs(var_formula) + 1e-18
     # deterministic truncation: the "expectation" is the single realisation, and it
     # misses exactly the dropped suffix
     mask, pi, cut = select(SEL_DET, cu, beta=0.5)
@@ -377,3 +385,62 @@ def test_general_cut_law_enumeration_is_unbiased():
             e_dW = e_dW + q[L - 1] * out["dW"]
         assert abs(e_loss - full["loss"]) < 2e-7 * abs(full["loss"]) + 1e-9
         np.testing.assert_allclose(e_dW, full["dW"], atol=2e-7 * np.abs(full["dW"]).max())
+
+
+def test_cutlaw_enumeration_is_unbiased():
+    """Proposition 1 under a non-uniform cut law given as masses q(l): weighting every cut by
+    its probability k_l / S_1 and using select_cutlaw's pi gives the full-token loss and dW."""
+    from oracle import cutlaw_counts
+    w, b = _tiny(old_noise=0.3, lengths=[6, 9, 5, 7, 4, 8, 3, 10], rewards=[1, 0, 0, 1, 0, 1, 0, 0])
+    cu = b["cu_seqlens"]
+    q = np.concatenate([0.85 ** np.arange(T) + 0.05 for T in np.diff(cu)]).astype(np.float32) / 16
+    _, pi, _ = select_cutlaw(cu, q, seed=0)
+    k = cutlaw_counts(q)
+    for i in range(w.B):
+        T = cu[i + 1] - cu[i]
+        kk = k[cu[i]:cu[i + 1]].astype(np.float64)
+        prob = kk / kk.sum()                          # Pr(L = l), l = 1..T
+        only = np.zeros(b["n_tot"], dtype=np.uint8)
+        only[cu[i]:cu[i + 1]] = 1
+        full = _run(b, only, np.ones_like(pi))
+        e_loss, e_dW = 0.0, 0.0
+        for L in range(1, T + 1):
+            m = np.zeros(b["n_tot"], dtype=np.uint8)
+            m[cu[i]:cu[i] + L] = 1
+            out = _run(b, m, pi)
+            e_loss += prob[L - 1] * out["loss"]
+            e_dW = e_dW + prob[L - 1] * out["dW"]
+        assert abs(e_loss - full["loss"]) < 2e-7 * abs(full["loss"]) + 1e-9
+        np.testing.assert_allclose(e_dW, full["dW"], atol=2e-7 * np.abs(full["dW"]).max())
+
+
+def test_dW_rows_match_full_dW_and_finite_differences():
+    w, b = _tiny(old_noise=0.3)
+    mask, pi, _ = select(SEL_URS, b["cu_seqlens"], p=0.5, seed=4)
+    si, sr, so, n = compact(mask, b["cu_seqlens"])
+    full = _run(b, mask, pi)
+    y = b["targets"][si]
+    v_ids = np.array([0, int(y[0]), int(y[n // 2]), 17, w.V - 1])
+    A = b["adv"].astype(np.float64)[sr]
+    g = grad_coeff(full["ratio"], A, full["w"], 0.2, 0.2)
+    H = b["hidden"][si]
+    blocks = [H[lo:lo + 37] for lo in range(0, n, 37)]          # streamed in ragged blocks
+    rows, dense = policy_loss_dW_rows(blocks, b["W"][v_ids], v_ids, y, g, full["lse"])
+    np.testing.assert_allclose(rows, full["dW"][v_ids], atol=1e-15 + 1e-12 * np.abs(full["dW"]).max())
+    np.testing.assert_allclose(dense, full["dW_dense"][v_ids],
+                               atol=1e-15 + 1e-12 * np.abs(full["dW_dense"]).max())
+    assert np.abs(rows - dense).max() > 0                       # target rows are in the sample
+
+    def loss_at(W):
+        return policy_loss_fwd(b["hidden"], W, b["targets"], b["old_logp"], b["adv"], pi,
+                               b["cu_seqlens"], si, sr)["loss"]
+    W0 = b["W"].astype(np.float64)
+    step = 1e-6
+    rng = np.random.default_rng(0)
+    for r, v in enumerate(v_ids):
+        j = int(rng.integers(w.d))
+        Wp, Wm = W0.copy(), W0.copy()
+        Wp[v, j] += step
+        Wm[v, j] -= step
+        fd = (loss_at(Wp) - loss_at(Wm)) / (2 * step)
+        assert abs(fd - rows[r, j]) < 1e-6 * np.abs(full["dW"]).max() + 1e-10

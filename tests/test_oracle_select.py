@@ -329,3 +329,111 @@ def test_gather_scatter_rows():
     s = scatter_rows(g, si, cu[-1])
     assert np.array_equal(s, x * mask[:, None])
     assert scatter_rows(g[:0], si[:0], 5).shape == (5, 6)
+
+
+# ------------------------------------------------------ sharding by response
+def test_resp_base_makes_a_shard_draw_the_whole_batch_masks():
+    """A shard that passes the global index of its first response realises, for its own
+    responses, exactly the mask, pi and cut the whole batch realises (Section 3.1: masks
+    of different responses are drawn independently, so this is what keeps Proposition 1
+    valid response by response under data-parallel sharding)."""
+    T = np.array([37, 0, 64, 21, 5, 90, 1, 12])
+    cu = _cu(T)
+    for mode, kw in ((SEL_URS, dict(p=0.5)), (SEL_RPC, dict(min_cut=4)), (SEL_DET, dict(beta=0.5))):
+        mask, pi, cut = select(mode, cu, seed=9, offset=3, **kw)
+        for lo, hi in ((0, 3), (3, 8), (5, 6)):
+            m2, p2, c2 = select(mode, _cu(T[lo:hi]), seed=9, offset=3, resp_base=lo, **kw)
+            assert np.array_equal(m2, mask[cu[lo]:cu[hi]])
+            assert np.array_equal(p2.view(np.uint32), pi[cu[lo]:cu[hi]].view(np.uint32))
+            if cut is not None:
+                assert np.array_equal(c2, cut[lo:hi])
+        # without the base the shard would reuse the draws of responses 0..: a different mask
+        if mode != SEL_DET:
+            m3, _, _ = select(mode, _cu(T[3:8]), seed=9, offset=3, **kw)
+            assert not np.array_equal(m3, mask[cu[3]:cu[8]])
+    surv = np.concatenate([_geometric_schedule(t, 0.9, 0.05) for t in T if t > 0])
+    ms, cs = select_survival(cu, surv, seed=2)
+    m2, c2 = select_survival(_cu(T[3:8]), surv[cu[3]:], seed=2, resp_base=3)
+    assert np.array_equal(m2, ms[cu[3]:]) and np.array_equal(c2, cs[3:])
+
+
+# ------------------------------------------------------------ general cut laws
+from oracle import cutlaw_counts, select_cutlaw  # noqa: E402
+
+
+def test_cutlaw_survival_is_the_suffix_sum_of_q():
+    """Eq. rpc-survival: p_t = sum_{l >= t} q(l), with p_1 = 1, p non-increasing and
+    p_T = q(T) > 0, for a geometric and a random law, against rational arithmetic."""
+    rng = np.random.default_rng(5)
+    T = np.array([1, 7, 64, 0, 300, 33])
+    cu = _cu(T)
+    q = np.concatenate([(np.maximum(0.9 ** np.arange(t), 0.02) * rng.uniform(0.5, 1.0, t)) / 40
+                        for t in T if t > 0])
+    q = q.astype(np.float32)
+    mask, pi, cut = select_cutlaw(cu, q, seed=1)
+    k = cutlaw_counts(q)
+    assert np.array_equal(k, np.floor(q.astype(np.float64) * 2.0 ** 32).astype(np.uint64))
+    for i, Ti in enumerate(T):
+        if Ti == 0:
+            assert cut[i] == 0
+            continue
+        p = pi[cu[i]:cu[i + 1]].astype(np.float64)
+        kk = [int(x) for x in k[cu[i]:cu[i + 1]]]
+        tot = sum(kk)
+        for t in range(Ti):
+            want = Fraction(sum(kk[t:]), tot)
+            assert abs(Fraction(float(p[t])) - want) <= want * Fraction(1, 2 ** 24)
+        assert p[0] == 1.0 and np.all(np.diff(p) <= 0) and p[-1] > 0
+        # and against the law itself: float32 rounding of pi plus the 2^-32 quantum of
+        # each of the (at most Ti) masses in the suffix
+        qq = q[cu[i]:cu[i + 1]].astype(np.float64)
+        np.testing.assert_allclose(p, np.cumsum(qq[::-1])[::-1] / qq.sum(), rtol=2e-7,
+                                   atol=2 * Ti * 2.0 ** -32 / qq.sum())
+        m = mask[cu[i]:cu[i + 1]]
+        assert 1 <= cut[i] <= Ti and m[:cut[i]].all() and not m[cut[i]:].any()
+
+
+def test_cutlaw_uniform_law_reproduces_the_uniform_cutoff_closed_form():
+    # q = 1/T on every position (T a power of two, so the masses are exact):
+    # pi_t = (T - t + 1) / T, bit for bit what the RPC mode writes for C = 1
+    for Tn in (8, 64, 4096):
+        cu = _cu([Tn, Tn])
+        _, pi, _ = select_cutlaw(cu, np.full(2 * Tn, 1.0 / Tn, dtype=np.float32))
+        _, pi_rpc, _ = select(SEL_RPC, cu, min_cut=1)
+        assert np.array_equal(pi.view(np.uint32), pi_rpc.view(np.uint32))
+    # a mandatory prefix C: zero mass before position C (App. B.2): pi = 1 for t <= C
+    Tn, C = 64, 16
+    q = np.zeros(Tn, dtype=np.float32)
+    q[C - 1:] = 1.0 / 64
+    _, pi, cut = select_cutlaw(_cu([Tn]), q, seed=3)
+    _, pi_rpc, _ = select(SEL_RPC, _cu([Tn]), min_cut=C)
+    assert np.array_equal(pi.view(np.uint32), pi_rpc.view(np.uint32)) and cut[0] >= C
+    # scaling the whole law changes nothing
+    _, pi2, cut2 = select_cutlaw(_cu([Tn]), q * np.float32(0.25), seed=3)
+    assert np.array_equal(pi2, pi) and cut2[0] == cut[0]
+    # no mass anywhere: the response is kept whole
+    m0, p0, c0 = select_cutlaw(_cu([5]), np.zeros(5, dtype=np.float32))
+    assert m0.all() and np.all(p0 == 1) and c0[0] == 5
+    # masses after the last positive one: those tokens are never selected (pi = 0)
+    m1, p1, c1 = select_cutlaw(_cu([4]), np.array([0.5, 0.5, 0.0, -1.0], dtype=np.float32))
+    assert np.all(p1[2:] == 0) and not m1[2:].any() and c1[0] in (1, 2)
+
+
+def test_cutlaw_draw_boundaries_and_frequencies():
+    """L >= t iff floor(u S_1 / 2^64) < S_t: checked against the integer draw recomputed
+    from the generator, and Pr(L = l) = q(l) over many responses (z-test, fixed seeds)."""
+    from oracle.philox import philox4x32_10 as ph
+    q = np.array([0.125, 0.25, 0.5, 0.125], dtype=np.float32)
+    k = [int(x) for x in cutlaw_counts(q)]
+    S = [sum(k[t:]) for t in range(4)]
+    for seed in range(300):
+        x0, x1, _, _ = ph(0, 7, 3, 0, seed, 0)
+        r = (((int(x1) << 32) | int(x0)) * S[0]) >> 64
+        want = sum(1 for t in range(4) if S[t] > r)
+        _, _, cut = select_cutlaw(_cu([4]), q, seed=seed, resp_base=7)
+        assert cut[0] == want
+    R = 6000
+    _, _, cuts = select_cutlaw(_cu([4] * R), np.tile(q, R), seed=13)
+    freq = np.bincount(cuts, minlength=5)[1:] / R
+    z = (freq - q) / np.sqrt(q * (1 - q) / R)
+    assert np.abs(z).max() < 4.5
