@@ -18,12 +18,19 @@
  *   - The library allocates no device memory: kernels that need scratch take
  *     a caller-provided `workspace` whose size the matching *_workspace_bytes
  *     function returns.  The workspace must be 256-byte aligned.
- *   - Return value: NAT_OK, or a negative nat_status; on error nothing was
- *     enqueued.  nat_last_error() gives a thread-local message.
+ *   - Return value: NAT_OK, or a negative nat_status.  Arguments are validated
+ *     (and the tensor maps of the bf16 path encoded) before the first
+ *     enqueue, so NAT_ERR_INVALID_ARG, NAT_ERR_UNSUPPORTED and NAT_ERR_CAPACITY
+ *     mean that nothing was enqueued; NAT_ERR_CUDA (a launch or memset refused
+ *     by the runtime) may leave earlier work of the same call on the stream.
+ *     nat_last_error() gives a thread-local message.
  *   - Device-side conditions that cannot be known at launch (a bounded wait
- *     that ran out, n_sel above the stated capacity) are recorded in the
- *     32-bit status word at the start of the workspace (see
- *     NAT_DEV_* bits); kernels never trap.
+ *     that ran out, n_sel above the stated capacity, a target outside the
+ *     vocabulary) are recorded in the 32-bit status word at the start of the
+ *     loss workspace (see NAT_DEV_* bits, nat_poll_status); kernels never trap.
+ *   - Alignment: mask, pi, surv and q arrays, the compacted lists and every
+ *     matrix must start on a 16-byte boundary (the kernels use 16-byte
+ *     accesses); a misaligned pointer is refused with NAT_ERR_INVALID_ARG.
  */
 #ifndef NAT_H_
 #define NAT_H_
@@ -48,10 +55,18 @@ typedef enum {
 #define NAT_DEV_CAPACITY 2u /* *n_sel exceeded n_sel_cap; surplus rows were ignored */
 #define NAT_DEV_FALLBACK 4u /* informational: nat_policy_loss_fwd_bwd redid some row chunk with
                                the two-pass kernels (results are valid) */
+#define NAT_DEV_BAD_TARGET 8u /* some selected token's target lies outside [0, V): that token
+                                 was left out (zero loss term and gradient, logp = NaN) */
 
 const char* nat_status_string(int status);
 const char* nat_last_error(void); /* host string, valid until the thread's next failing call */
 int nat_version(void);
+
+/* Copies the device status word at the head of a loss workspace to *host_word (host
+ * pointer) and waits for `stream`, i.e. for the loss calls enqueued on it so far.  (A
+ * convenience of this library; the paper has no counterpart.)  The word is the OR of the
+ * NAT_DEV_* bits raised by the last loss call that used the workspace. */
+int nat_poll_status(const void* workspace, void* stream, uint32_t* host_word);
 
 /* ---------------------------------------------------------------------------
  * Group-relative advantage (Eq. grpo-adv, Section 2.2):
@@ -67,7 +82,8 @@ int nat_grpo_adv(int32_t P, int32_t G, const float* rewards, float eps, float* a
  * Token selection (Section 3.1 "Random masking", URS; Section 4 RPC with the
  * uniform and minimum-cutoff laws; deterministic truncation as the biased
  * comparison).  Random draws are Philox4x32-10 outputs, a pure function of
- * (seed, offset, response index, position):
+ * (seed, offset, response index, position); below i stands for resp_base + the
+ * response's index in cu_seqlens:
  *   key     = (seed_lo, seed_hi ^ offset_hi)
  *   URS     token t uses word (t-1)%4 of counter ((t-1)/4, i, 0, offset_lo);
  *           m = [x < thr], thr = clamp(floor(p 2^32), 1, 2^32), pi = thr/2^32.
@@ -81,8 +97,12 @@ int nat_grpo_adv(int32_t P, int32_t G, const float* rewards, float eps, float* a
  * (L_i or K_i, 0 for an empty response; may be NULL for URS, which leaves it
  * untouched).  cu_seqlens int32 [B+1] on the device; n_tot is the host's copy
  * of cu_seqlens[B].  T_i = 0 is allowed.
+ * resp_base: index, in the whole job's batch, of the first response of cu_seqlens.  A
+ * data-parallel rank that holds responses [lo, hi) of the batch passes its own cu_seqlens
+ * and resp_base = lo and realises exactly the masks the whole batch would (masks of
+ * different responses are independent, Section 3.1); 0 for an unsharded batch.
  * Errors: NAT_ERR_INVALID_ARG for p outside (0,1], beta outside (0,1],
- * min_cut < 0, B < 0, n_tot < 0 or null pointers.
+ * min_cut < 0, B < 0, n_tot < 0, resp_base < 0, null or misaligned pointers.
  * ------------------------------------------------------------------------- */
 typedef enum { NAT_SEL_URS = 0, NAT_SEL_RPC = 1, NAT_SEL_DET = 2 } nat_sel_mode;
 
@@ -93,6 +113,8 @@ typedef struct {
   double beta;     /* DET: kept fraction in (0,1] */
   uint64_t seed;
   uint64_t offset; /* caller's step counter: a new offset gives fresh draws */
+  int32_t resp_base; /* global index of the first response (0 unless the batch is a shard) */
+  int32_t reserved;  /* set to 0 */
 } nat_select_params;
 
 int nat_select(const nat_select_params* params /* host */, int32_t B, const int32_t* cu_seqlens,
@@ -105,19 +127,43 @@ int nat_select(const nat_select_params* params /* host */, int32_t B, const int3
  *   surv float32 [n_tot]: p_{i,t} = Pr(L_i >= t) for every packed token; inside a
  *   response it must start at 1, never increase and stay positive (not checked).
  * Response i draws u = (x0 >> 8) 2^-24 from the Philox block with counter
- * (0, i, 2, offset_lo), key as in nat_select; m_t = [u < surv], a prefix of
+ * (0, resp_base + i, 2, offset_lo), key as in nat_select; m_t = [u < surv], a prefix of
  * length L_i because surv is monotone, and Pr(L_i >= t) = ceil(surv 2^24) / 2^24.
  * Outputs: mask uint8 [n_tot], cut_len int32 [B] (L_i; 0 for an empty response).
  * The inclusion probabilities are the schedule: pass `surv` as `pi` to the loss.
  * surv and mask must be 16-byte aligned.
  * ------------------------------------------------------------------------- */
 int nat_select_survival(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const float* surv,
-                        uint64_t seed, uint64_t offset, uint8_t* mask, int32_t* cut_len,
-                        void* stream);
+                        uint64_t seed, uint64_t offset, int32_t resp_base, uint8_t* mask,
+                        int32_t* cut_len, void* stream);
 
 /* ---------------------------------------------------------------------------
- * Compaction of the selected tokens ("only included tokens contribute to
- * backpropagation", Section 1; Eq. ht-estimator sums over m = 1 only).
+ * Random Prefix Cutting under a caller-given cut law (Section 4: Eq. rpc-mask; the
+ * survival function is the suffix sum of the law, Eq. rpc-survival; Appendix B.3 on laws
+ * other than the uniform one).
+ *   q float32 [n_tot]: the mass q_i(l) the law of token n's response puts on cutting right
+ *   after that token, up to a common positive factor per response.  Masses enter in
+ *   32-bit fixed point, k = floor(min(q, 1) 2^32) for q > 0 and 0 otherwise, so that every
+ *   sum below is an exact 64-bit integer, independent of the order of summation:
+ *     S_t  = sum_{l >= t} k_l       (a scan over the packed stream on the device)
+ *     pi_t = float32(double(S_t) / double(S_1)):  pi_1 = 1 and pi never increases, by
+ *            construction; pi_t > 0 wherever the law still has mass at or after t
+ *     u    = x1 2^32 + x0 of the Philox block with counter (0, resp_base + i, 3, offset_lo),
+ *     r    = floor(u S_1 / 2^64),  m_t = [S_t > r]:  L_i = max{t : S_t > r},
+ *            Pr(L_i >= t) = S_t / S_1 to within S_1 2^-64.
+ *   A response whose masses are all zero is kept whole with pi = 1.  Tokens after the
+ *   last positive mass get pi = 0 and are never selected.
+ * Outputs: mask uint8 [n_tot], pi float32 [n_tot], cut_len int32 [B].
+ * workspace: nat_select_cutlaw_workspace_bytes(B, n_tot) bytes, 256-byte aligned.
+ * ------------------------------------------------------------------------- */
+size_t nat_select_cutlaw_workspace_bytes(int32_t B, int64_t n_tot);
+int nat_select_cutlaw(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const float* q,
+                      uint64_t seed, uint64_t offset, int32_t resp_base, uint8_t* mask, float* pi,
+                      int32_t* cut_len, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Compaction of the selected tokens (Section 1: tokens that were not selected take no
+ * part in the backward pass; Eq. ht-estimator sums over m = 1 only).
  *   sel_idx  int32 [cap]   ascending packed indices n with mask[n] != 0
  *   sel_resp int32 [cap]   resp(sel_idx[k])
  *   sel_offsets int32 [B+1] number of selected tokens in responses < i
@@ -132,9 +178,24 @@ int nat_compact(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8
                 int64_t cap, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
- * Packing for prefix-truncated computation (Section 4, "Compute savings: prefix
- * structure enables true forward truncation": under RPC the model only has to
- * process the prefix 1..L_i of each response).
+ * Compaction under a prefix mask (Eq. rpc-mask: m_t = 1[t <= L_i]; also the deterministic
+ * truncation).  The selected tokens of response i are the packed indices
+ * [cu_seqlens[i], cu_seqlens[i] + L_i), so the lists follow from cut_len alone: the mask
+ * is not read and nothing but the lists is written (8 bytes per selected token).
+ *   cut_len int32 [B]: L_i as written by nat_select (RPC, DET), nat_select_survival or
+ *   nat_select_cutlaw; values are clamped to [0, T_i].
+ * Outputs and capacity rule as for nat_compact; the results are identical to
+ * nat_compact on the corresponding mask.  n_tot (host copy of cu_seqlens[B]) bounds the
+ * launch.  No workspace.
+ * ------------------------------------------------------------------------- */
+int nat_compact_prefix(int32_t B, const int32_t* cu_seqlens, int64_t n_tot,
+                       const int32_t* cut_len, int32_t* sel_idx, int32_t* sel_resp,
+                       int32_t* sel_offsets, int32_t* n_sel, int64_t cap, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Packing for prefix-truncated computation (Section 4, the paragraph on compute
+ * savings: under RPC the model only has to process the prefix 1..L_i of each
+ * response, forward as well as backward).
  *   nat_gather_rows   dst[k, :] = src[sel_idx[k], :]  for k < min(*n_sel, cap)
  *   nat_scatter_rows  dst = 0 over [n_tot, row_bytes], then
  *                     dst[sel_idx[k], :] = src[k, :]   (e.g. compact dHidden back
@@ -193,11 +254,17 @@ int nat_compact_static(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, cons
  *
  * dtype NAT_BF16: hidden, W, dHidden are bfloat16 and the projection runs on
  * the tensor cores; requires d % 64 == 0.  dtype NAT_F32: float32 operands,
- * plain fp32 arithmetic, any d and V (meant for small problems).
+ * plain fp32 arithmetic, any V and d <= 1024 (meant for small problems; a larger d is
+ * refused with NAT_ERR_UNSUPPORTED and has workspace size 0).
  * hidden is [n_tot, d] row-major (row sel_idx[k] is used) or, with
  * hidden_is_compact, [>= n_sel, d] with row k belonging to sel_idx[k].
  * W is [V, d] row-major.  targets int32 [n_tot] in [0, V); old_logp, pi
- * float32 [n_tot]; adv float32 [B].  n_sel is the device scalar written by
+ * float32 [n_tot]; adv float32 [number of responses in cu_seqlens].  params->B is the
+ * divisor of the batch mean: the number of responses of the WHOLE job's batch, which
+ * exceeds the number of responses passed here when the batch is sharded over
+ * data-parallel ranks (the ranks' losses and dW then add up to the job's).
+ * A target outside [0, V) raises NAT_DEV_BAD_TARGET and its token is left out.
+ * n_sel is the device scalar written by
  * nat_compact; n_sel_cap is a host upper bound on it (grid and workspace are
  * sized from it; rows beyond it are ignored and NAT_DEV_CAPACITY is raised).
  * Outputs: loss float32 device scalar; logp, lse float32 [n_sel_cap] (entries
@@ -213,7 +280,7 @@ typedef struct {
   int32_t d;
   int32_t V;
   int32_t dtype; /* NAT_F32 | NAT_BF16 */
-  int32_t B;     /* number of responses (the batch mean's divisor) */
+  int32_t B;     /* number of responses of the whole batch (the batch mean's divisor) */
   float clip_lo; /* ratio is clipped to [1-clip_lo, 1+clip_hi] */
   float clip_hi;
   int32_t hidden_is_compact;
@@ -245,6 +312,9 @@ int nat_policy_loss_fwd(const nat_loss_params* params /* host */, const void* hi
  * logp and lse are the forward's outputs.  dloss is a device float scalar
  * (NULL means 1).  dHidden has hidden's dtype, [n_sel_cap, d]; rows >= n_sel
  * are not written.  With accumulate_dW the product is added to dW's contents.
+ * Every element of dHidden and dW is summed in a fixed order (tokens that share a target
+ * are added to that row of dW in ascending order), so a call repeated on the same inputs
+ * reproduces its outputs bit for bit.
  * ------------------------------------------------------------------------- */
 int nat_policy_loss_bwd(const nat_loss_params* params /* host */, const void* hidden,
                         const void* W, const int32_t* targets, const float* old_logp,

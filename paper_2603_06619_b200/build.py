@@ -7,7 +7,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnat_b200.so")
-SOURCES = ["nat_api.cu", "nat_token.cu", "nat_select.cu", "nat_loss_f32.cu", "nat_loss_bf16.cu"]
+SOURCES = ["nat_api.cu", "nat_token.cu", "nat_select.cu", "nat_prefix.cu", "nat_loss_f32.cu",
+           "nat_loss_bf16.cu"]
 
 
 def _stale():

@@ -56,6 +56,9 @@ static int validate(const char* who, const nat_loss_params* p, const LossArgs& a
       return fail(NAT_ERR_INVALID_ARG, "%s: matrices must be 16-byte aligned", who);
   }
   const size_t need = nat_policy_loss_workspace_bytes(p, a.cap);
+  if (need == 0)
+    return fail(NAT_ERR_UNSUPPORTED, "%s: this dtype does not cover d = %d (float32 needs d <= 1024)",
+                who, p->d);
   if (!a.workspace || a.workspace_bytes < need)
     return fail(NAT_ERR_CAPACITY, "%s: workspace too small (%zu < %zu)", who, a.workspace_bytes,
                 need);
@@ -81,7 +84,16 @@ const char* nat_status_string(int status) {
 
 const char* nat_last_error(void) { return nat::error_buffer(); }
 
-int nat_version(void) { return 1; }
+int nat_version(void) { return 2; }
+
+int nat_poll_status(const void* workspace, void* stream, uint32_t* host_word) {
+  if (!workspace || !host_word)
+    return nat::fail(NAT_ERR_INVALID_ARG, "nat_poll_status: null pointer");
+  NAT_CUDA(cudaMemcpyAsync(host_word, workspace, sizeof(uint32_t), cudaMemcpyDeviceToHost,
+                           (cudaStream_t)stream));
+  NAT_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  return NAT_OK;
+}
 
 size_t nat_policy_loss_workspace_bytes(const nat_loss_params* p, int64_t n_sel_cap) {
   if (!p || n_sel_cap < 0 || p->d <= 0 || p->V <= 0) return 0;

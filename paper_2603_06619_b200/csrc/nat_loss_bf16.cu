@@ -443,6 +443,9 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
           row_ok = k < n_valid;
           if (row_ok) {
             if (MODE == kFwd || MODE == kDh || MODE == kE) y = p.targets[p.sel_idx[k]];
+            // a target outside the vocabulary has g = 0 (its token is left out); keep the
+            // one-hot row read in bounds
+            if (MODE == kDh && (unsigned)y >= (unsigned)p.V) y = 0;
             if (MODE == kDz || MODE == kDh) gk = p.g[k];
             if (MODE == kDz) lk = p.lse[k];
             if (MODE == kE) lk = p.mref[k];
@@ -743,7 +746,7 @@ __global__ void fwd_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_se
     for (int sp = 0; sp < n_splits; ++sp)
       S += part_s[(size_t)sp * cap_pad + k] * expf(part_m[(size_t)sp * cap_pad + k] - M);
     const float l = M + logf(S);
-    const float lp = zt[k] - l;
+    const float lp = target_ok(c, k) ? zt[k] - l : __int_as_float(0x7FC00000);
     lse[k] = l;
     logp[k] = lp;
     float t, g;
@@ -783,7 +786,7 @@ __global__ void fused_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_
         float S = 0.f;
         for (int sp = 0; sp < n_splits; ++sp) S += part_s[(size_t)sp * cap_pad + k];
         const float l = mref[k] + logf(S);
-        const float lp = zt[k] - l;
+        const float lp = target_ok(c, k) ? zt[k] - l : __int_as_float(0x7FC00000);
         lse[k] = l;
         logp[k] = lp;
         float t, g;
@@ -824,36 +827,135 @@ __global__ void note_fallback_kernel(const int32_t* __restrict__ ovf, int n_chun
     if (ovf[c] != 0) atomicOr(status, NAT_DEV_FALLBACK);
 }
 
-// One-hot part of dW: dW[y_k, :] += g_k h_k.  Tokens that share a target meet
-// in the same row, hence atomics.
-__global__ void onehot_dw_kernel(const __nv_bfloat16* __restrict__ Hc,
-                                 const int32_t* __restrict__ targets,
-                                 const int32_t* __restrict__ sel_idx, const float* __restrict__ g,
-                                 const int32_t* __restrict__ n_sel, int cap, int d,
-                                 float* __restrict__ dW) {
+// One-hot part of dW: dW[y_k, :] += g_k h_k.  Tokens that share a target meet in the same
+// row of dW; to keep the sum's order fixed (and with it the bits of dW) the tokens are first
+// grouped by target, each group sorted by token index, and every row then receives its
+// tokens in ascending order from a single thread per column:
+//   count   tokens per target (integer atomics: the counts do not depend on their order)
+//   scan    exclusive scan of the counts over the vocabulary -> group offsets
+//   fill    every token takes a slot of its group (the slot order is arbitrary)
+//   rank    every token counts the smaller indices of its group -> its sorted position
+//   apply   one block per target and 1024-column slice walks the sorted group
+__global__ void onehot_count_kernel(const int32_t* __restrict__ targets,
+                                    const int32_t* __restrict__ sel_idx,
+                                    const float* __restrict__ g, const int32_t* __restrict__ n_sel,
+                                    int cap, int V, int32_t* __restrict__ count) {
   int n = *n_sel;
   n = n < cap ? n : cap;
-  for (int k = blockIdx.x; k < n; k += gridDim.x) {
-    const float gk = g[k];
-    if (gk == 0.f) continue;
+  for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
+    if (g[k] == 0.f) continue;
     const int y = targets[sel_idx[k]];
-    const uint2* h = reinterpret_cast<const uint2*>(Hc + (size_t)k * d);  // four bf16 at a time
-    float* dst = dW + (size_t)y * d;
-    for (int j = threadIdx.x; j < d / 4; j += blockDim.x) {
-      const uint2 hv = h[j];
-      const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&hv.x);
-      const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&hv.y);
-      tc::red_add_f32x4(dst + 4 * j, gk * __low2float(lo), gk * __high2float(lo),
-                        gk * __low2float(hi), gk * __high2float(hi));
+    if ((unsigned)y < (unsigned)V) atomicAdd(&count[y], 1);
+  }
+}
+
+// off[v] = number of tokens whose target is below v (off[V] = all of them); the counts are
+// cleared on the way so that they can serve as the groups' fill cursors.
+__global__ void __launch_bounds__(1024)
+onehot_scan_kernel(int32_t* __restrict__ count, int V, int32_t* __restrict__ off) {
+  __shared__ int warp_tot[2][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int carry = 0;
+  for (int base = 0, tile = 0; base < V; base += 4096, ++tile) {
+    const int v0 = base + (int)threadIdx.x * 4;
+    int c[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      c[e] = v0 + e < V ? count[v0 + e] : 0;
+      if (v0 + e < V) count[v0 + e] = 0;
     }
+    const int sum = c[0] + c[1] + c[2] + c[3];
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    int* tot = warp_tot[tile & 1];
+    if (lane == 31) tot[warp] = incl;
+    __syncthreads();
+    const int wt = tot[lane];
+    int wincl = wt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xFFFFFFFFu, wincl, o);
+      if (lane >= o) wincl += up;
+    }
+    const int tile_total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
+    const int warp_excl = __shfl_sync(0xFFFFFFFFu, wincl - wt, warp);
+    int e0 = carry + warp_excl + incl - sum;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (v0 + e < V) off[v0 + e] = e0;
+      e0 += c[e];
+    }
+    carry += tile_total;
+  }
+  if (threadIdx.x == 0) off[V] = carry;
+}
+
+__global__ void onehot_fill_kernel(const int32_t* __restrict__ targets,
+                                   const int32_t* __restrict__ sel_idx,
+                                   const float* __restrict__ g, const int32_t* __restrict__ n_sel,
+                                   int cap, int V, const int32_t* __restrict__ off,
+                                   int32_t* __restrict__ cursor, int32_t* __restrict__ list) {
+  int n = *n_sel;
+  n = n < cap ? n : cap;
+  for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
+    if (g[k] == 0.f) continue;
+    const int y = targets[sel_idx[k]];
+    if ((unsigned)y < (unsigned)V) list[off[y] + atomicAdd(&cursor[y], 1)] = k;
+  }
+}
+
+__global__ void onehot_rank_kernel(const int32_t* __restrict__ targets,
+                                   const int32_t* __restrict__ sel_idx, int V,
+                                   const int32_t* __restrict__ off,
+                                   const int32_t* __restrict__ list,
+                                   int32_t* __restrict__ sorted) {
+  const int n_live = off[V];
+  for (int p = blockIdx.x * blockDim.x + threadIdx.x; p < n_live; p += gridDim.x * blockDim.x) {
+    const int k = list[p];
+    const int y = targets[sel_idx[k]];
+    const int lo = off[y], hi = off[y + 1];
+    int rank = 0;
+    for (int j = lo; j < hi; ++j) rank += list[j] < k ? 1 : 0;
+    sorted[lo + rank] = k;
+  }
+}
+
+// blockIdx.y selects a slice of 1024 columns (four per thread); rows are taken grid-stride.
+__global__ void __launch_bounds__(256)
+onehot_apply_kernel(const __nv_bfloat16* __restrict__ Hc, const float* __restrict__ g, int V,
+                    int d, const int32_t* __restrict__ off, const int32_t* __restrict__ sorted,
+                    float* __restrict__ dW) {
+  const int col = (blockIdx.y * 256 + threadIdx.x) * 4;
+  if (col >= d) return;
+  for (int y = blockIdx.x; y < V; y += gridDim.x) {
+    const int lo = off[y], hi = off[y + 1];
+    if (lo == hi) continue;
+    float* dst = dW + (size_t)y * d + col;
+    float4 acc = *reinterpret_cast<const float4*>(dst);
+    for (int e = lo; e < hi; ++e) {
+      const int k = sorted[e];
+      const float gk = g[k];
+      const uint2 hv = *reinterpret_cast<const uint2*>(Hc + (size_t)k * d + col);
+      const __nv_bfloat162 h01 = *reinterpret_cast<const __nv_bfloat162*>(&hv.x);
+      const __nv_bfloat162 h23 = *reinterpret_cast<const __nv_bfloat162*>(&hv.y);
+      acc.x = fmaf(gk, __low2float(h01), acc.x);
+      acc.y = fmaf(gk, __high2float(h01), acc.y);
+      acc.z = fmaf(gk, __low2float(h23), acc.z);
+      acc.w = fmaf(gk, __high2float(h23), acc.w);
+    }
+    *reinterpret_cast<float4*>(dst) = acc;
   }
 }
 
 // ------------------------------------------------------------- host side
 struct Layout {
   int cap_pad, n_tiles, n_splits, chunk_rows, n_chunks, ldz;
-  size_t off_term, off_g, off_zt, off_pm, off_ps, off_mref, off_cs, off_ovf, off_prog, off_hc,
-      off_hs, off_dz, total;
+  size_t off_term, off_g, off_zt, off_pm, off_ps, off_mref, off_cs, off_ovf, off_prog, off_ohc,
+      off_oho, off_ohl, off_ohs, off_hc, off_hs, off_dz, total;
 };
 
 // Number of vocabulary splits.  A work unit of the vocabulary sweeps is (block of rows,
@@ -912,6 +1014,10 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   L.off_cs = take(sizeof(float) * L.cap_pad);
   L.off_ovf = take(sizeof(int32_t) * L.n_chunks);
   L.off_prog = take(sizeof(unsigned long long) * kMaxPairs);
+  L.off_ohc = take(sizeof(int32_t) * (size_t)p.V);
+  L.off_oho = take(sizeof(int32_t) * ((size_t)p.V + 1));
+  L.off_ohl = take(sizeof(int32_t) * L.cap_pad);
+  L.off_ohs = take(sizeof(int32_t) * L.cap_pad);
   off = align_up(off, 1024);
   L.off_hc = take(sizeof(__nv_bfloat16) * (size_t)L.cap_pad * p.d);
   L.off_hs = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * p.d);
@@ -1126,28 +1232,12 @@ int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2
   return launch_tc_impl<MODE, 1, 1>(a, b1, c, q, m_blocks128 * per_block, stream);
 }
 
-TokenCtx make_ctx(const LossArgs& a) {
-  TokenCtx c;
-  c.targets = a.targets;
-  c.old_logp = a.old_logp;
-  c.adv = a.adv;
-  c.pi = a.pi;
-  c.cu_seqlens = a.cu_seqlens;
-  c.sel_idx = a.sel_idx;
-  c.sel_resp = a.sel_resp;
-  c.B = a.p.B;
-  c.clip_lo = a.p.clip_lo;
-  c.clip_hi = a.p.clip_hi;
-  c.kl_beta = a.p.kl_beta;
-  c.ref_logp = a.p.ref_logp;
-  return c;
-}
-
 struct Ws {
   WorkspaceHead* head;
   float *term, *g, *zt, *pm, *ps, *mref, *cs;
   int32_t* ovf;
   unsigned long long* prog;
+  int32_t *oh_count, *oh_off, *oh_list, *oh_sorted;  // grouping of the tokens by target
   __nv_bfloat16 *hc, *hs, *dz;
 };
 
@@ -1164,6 +1254,10 @@ Ws carve(void* ws, const Layout& L) {
   w.cs = reinterpret_cast<float*>(b + L.off_cs);
   w.ovf = reinterpret_cast<int32_t*>(b + L.off_ovf);
   w.prog = reinterpret_cast<unsigned long long*>(b + L.off_prog);
+  w.oh_count = reinterpret_cast<int32_t*>(b + L.off_ohc);
+  w.oh_off = reinterpret_cast<int32_t*>(b + L.off_oho);
+  w.oh_list = reinterpret_cast<int32_t*>(b + L.off_ohl);
+  w.oh_sorted = reinterpret_cast<int32_t*>(b + L.off_ohs);
   w.hc = reinterpret_cast<__nv_bfloat16*>(b + L.off_hc);
   w.hs = reinterpret_cast<__nv_bfloat16*>(b + L.off_hs);
   w.dz = reinterpret_cast<__nv_bfloat16*>(b + L.off_dz);
@@ -1219,7 +1313,7 @@ struct Maps {
   CUtensorMap dwRed;  // dW as a reduction target (valid only when the call has a dW)
 };
 
-int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
+int encode_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
   int s;
   const uint64_t dpitch = (uint64_t)a.p.d * 2, zpitch = (uint64_t)L.ldz * 2;
   if ((s = make_map(&m->hcK, w.hc, a.p.d, L.cap_pad, dpitch, BK, BM)) != NAT_OK) return s;
@@ -1233,6 +1327,45 @@ int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
   if ((s = make_map(&m->dzSt, w.dz, a.p.V, L.chunk_rows, zpitch, 64, 32)) != NAT_OK) return s;
   m->dwRed = m->dzSt;
   if (a.dW != nullptr && (s = make_map_f32(&m->dwRed, a.dW, a.p.d, a.p.V)) != NAT_OK) return s;
+  return NAT_OK;
+}
+
+// The tensor maps depend only on the operands' addresses and shapes, which a trainer keeps
+// from step to step, so the last few sets are remembered (encoding ten maps costs tens of
+// microseconds of host time per call, a visible share of a small head's step).
+struct MapsKey {
+  const void *ws, *W, *dW;
+  int d, V, cap_pad, chunk_rows, ldz, dev;
+  bool operator==(const MapsKey& o) const {
+    return ws == o.ws && W == o.W && dW == o.dW && d == o.d && V == o.V &&
+           cap_pad == o.cap_pad && chunk_rows == o.chunk_rows && ldz == o.ldz && dev == o.dev;
+  }
+};
+constexpr int kMapsCached = 8;
+std::mutex g_maps_mutex;
+MapsKey g_maps_key[kMapsCached];
+Maps g_maps_val[kMapsCached];
+bool g_maps_used[kMapsCached] = {false};
+int g_maps_next = 0;
+
+int make_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
+  MapsKey key{a.workspace, a.W, a.dW, a.p.d, a.p.V, L.cap_pad, L.chunk_rows, L.ldz, 0};
+  int s = current_device(&key.dev);
+  if (s != NAT_OK) return s;
+  {
+    std::lock_guard<std::mutex> lock(g_maps_mutex);
+    for (int i = 0; i < kMapsCached; ++i)
+      if (g_maps_used[i] && g_maps_key[i] == key) {
+        *m = g_maps_val[i];
+        return NAT_OK;
+      }
+  }
+  if ((s = encode_maps(a, L, w, m)) != NAT_OK) return s;
+  std::lock_guard<std::mutex> lock(g_maps_mutex);
+  g_maps_key[g_maps_next] = key;
+  g_maps_val[g_maps_next] = *m;
+  g_maps_used[g_maps_next] = true;
+  g_maps_next = (g_maps_next + 1) % kMapsCached;
   return NAT_OK;
 }
 
@@ -1260,10 +1393,23 @@ int launch_two_pass_chunk(const LossArgs& a, const Layout& L, const Ws& w, const
 }
 
 int launch_onehot(const LossArgs& a, const Ws& w) {
-  const int grid = (int)(a.cap < 8192 ? a.cap : 8192);
-  onehot_dw_kernel<<<grid, 256, 0, a.stream>>>(w.hc, a.targets, a.sel_idx, w.g, a.n_sel,
-                                               (int)a.cap, a.p.d, a.dW);
-  NAT_LAUNCH_CHECK("onehot_dw_kernel");
+  const int V = a.p.V, d = a.p.d, cap = (int)a.cap;
+  const int tok_grid = (int)((a.cap + 255) / 256 < 1184 ? (a.cap + 255) / 256 : 1184);
+  NAT_CUDA(cudaMemsetAsync(w.oh_count, 0, sizeof(int32_t) * (size_t)V, a.stream));
+  onehot_count_kernel<<<tok_grid, 256, 0, a.stream>>>(a.targets, a.sel_idx, w.g, a.n_sel, cap, V,
+                                                     w.oh_count);
+  NAT_LAUNCH_CHECK("onehot_count_kernel");
+  onehot_scan_kernel<<<1, 1024, 0, a.stream>>>(w.oh_count, V, w.oh_off);
+  NAT_LAUNCH_CHECK("onehot_scan_kernel");
+  onehot_fill_kernel<<<tok_grid, 256, 0, a.stream>>>(a.targets, a.sel_idx, w.g, a.n_sel, cap, V,
+                                                    w.oh_off, w.oh_count, w.oh_list);
+  NAT_LAUNCH_CHECK("onehot_fill_kernel");
+  onehot_rank_kernel<<<tok_grid, 256, 0, a.stream>>>(a.targets, a.sel_idx, V, w.oh_off, w.oh_list,
+                                                    w.oh_sorted);
+  NAT_LAUNCH_CHECK("onehot_rank_kernel");
+  const dim3 grid((unsigned)(V < 8192 ? V : 8192), (unsigned)((d + 1023) / 1024), 1);
+  onehot_apply_kernel<<<grid, 256, 0, a.stream>>>(w.hc, w.g, V, d, w.oh_off, w.oh_sorted, a.dW);
+  NAT_LAUNCH_CHECK("onehot_apply_kernel");
   return NAT_OK;
 }
 
@@ -1278,12 +1424,12 @@ int loss_bf16_fwd(const LossArgs& a) {
   if (s != NAT_OK) return s;
   const Layout L = make_layout(a.p, a.cap);
   const Ws w = carve(a.workspace, L);
+  Maps m;  // encoded before anything is enqueued: a refusal leaves the stream untouched
+  if (a.cap > 0 && (s = make_maps(a, L, w, &m)) != NAT_OK) return s;
   NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
-  const TokenCtx c = make_ctx(a);
+  const TokenCtx c = make_token_ctx(a, &w.head->status);
   if (a.cap > 0) {
     if ((s = gather(a, L, w)) != NAT_OK) return s;
-    Maps m;
-    if ((s = make_maps(a, L, w, &m)) != NAT_OK) return s;
     const TcParams p = base_params(a, L, w);
     if ((s = launch_tc<kFwd>(m.hcK, m.wK, m.wK2, m.hcK, p, L.cap_pad / BM, L.n_splits, a.stream)) !=
         NAT_OK)
@@ -1301,15 +1447,15 @@ int loss_bf16_bwd(const LossArgs& a) {
   if (s != NAT_OK) return s;
   const Layout L = make_layout(a.p, a.cap);
   const Ws w = carve(a.workspace, L);
+  Maps m;
+  if (a.cap > 0 && (s = make_maps(a, L, w, &m)) != NAT_OK) return s;
   NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
   if (!a.p.accumulate_dW)
     NAT_CUDA(cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)a.p.V * a.p.d, a.stream));
   if (a.cap == 0) return NAT_OK;
-  const TokenCtx c = make_ctx(a);
+  const TokenCtx c = make_token_ctx(a, &w.head->status);
   if ((s = gather(a, L, w)) != NAT_OK) return s;
   if ((s = launch_grad_coeff(c, a.logp, a.n_sel, a.cap, a.dloss, w.g, a.stream)) != NAT_OK) return s;
-  Maps m;
-  if ((s = make_maps(a, L, w, &m)) != NAT_OK) return s;
   for (int row0 = 0; row0 < L.cap_pad; row0 += L.chunk_rows)
     if ((s = launch_two_pass_chunk(a, L, w, m, row0, nullptr)) != NAT_OK) return s;
   return launch_onehot(a, w);
@@ -1321,15 +1467,15 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
   if (s != NAT_OK) return s;
   const Layout L = make_layout(a.p, a.cap);
   const Ws w = carve(a.workspace, L);
+  Maps m;
+  if (a.cap > 0 && (s = make_maps(a, L, w, &m)) != NAT_OK) return s;
   NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
   NAT_CUDA(cudaMemsetAsync(w.ovf, 0, sizeof(int32_t) * L.n_chunks, a.stream));
   if (!a.p.accumulate_dW)
     NAT_CUDA(cudaMemsetAsync(a.dW, 0, sizeof(float) * (size_t)a.p.V * a.p.d, a.stream));
-  const TokenCtx c = make_ctx(a);
+  const TokenCtx c = make_token_ctx(a, &w.head->status);
   if (a.cap > 0) {
     if ((s = gather(a, L, w)) != NAT_OK) return s;
-    Maps m;
-    if ((s = make_maps(a, L, w, &m)) != NAT_OK) return s;
     const int mb = L.chunk_rows / BM;
     const int nb_d = (a.p.d + BN - 1) / BN;
     // Row references: the row maximum over the first vocabulary tile (a kFwd launch that

@@ -83,7 +83,8 @@ f32_fwd_kernel(TokenCtx c, const float* __restrict__ hidden, const float* __rest
       for (int w = 0; w < kWarps; ++w)
         if (s_s[w] > 0.f) S += s_s[w] * expf(m_s[w] - M);
       const float l = M + logf(S);
-      const float lp = zt_s[y % kWarps] - l;
+      const bool y_ok = (unsigned)y < (unsigned)V;
+      const float lp = y_ok ? zt_s[y % kWarps] - l : __int_as_float(0x7FC00000);
       lse[k] = l;
       logp[k] = lp;
       float t, g;
@@ -188,23 +189,6 @@ f32_dw_kernel(TokenCtx c, const float* __restrict__ hidden, const float* __restr
   }
 }
 
-TokenCtx make_ctx(const LossArgs& a) {
-  TokenCtx c;
-  c.targets = a.targets;
-  c.old_logp = a.old_logp;
-  c.adv = a.adv;
-  c.pi = a.pi;
-  c.cu_seqlens = a.cu_seqlens;
-  c.sel_idx = a.sel_idx;
-  c.sel_resp = a.sel_resp;
-  c.B = a.p.B;
-  c.clip_lo = a.p.clip_lo;
-  c.clip_hi = a.p.clip_hi;
-  c.kl_beta = a.p.kl_beta;
-  c.ref_logp = a.p.ref_logp;
-  return c;
-}
-
 int check_shape(const LossArgs& a) {
   if (a.p.d > kMaxD)
     return fail(NAT_ERR_UNSUPPORTED, "the fp32 path supports d <= %d (d = %d)", kMaxD, a.p.d);
@@ -213,7 +197,8 @@ int check_shape(const LossArgs& a) {
 
 }  // namespace
 
-size_t loss_f32_workspace_bytes(const nat_loss_params&, int64_t cap) {
+size_t loss_f32_workspace_bytes(const nat_loss_params& p, int64_t cap) {
+  if (p.d > kMaxD) return 0;  // not supported: see check_shape
   return sizeof(WorkspaceHead) + 2 * align_up(sizeof(float) * (size_t)cap, 256);
 }
 
@@ -222,7 +207,7 @@ int loss_f32_fwd(const LossArgs& a) {
   if (s != NAT_OK) return s;
   F32Ws w = carve(a.workspace, a.cap);
   NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
-  const TokenCtx c = make_ctx(a);
+  const TokenCtx c = make_token_ctx(a, &w.head->status);
   if (a.cap > 0) {
     const int grid = (int)min((int64_t)4096, a.cap);
     f32_fwd_kernel<<<grid, kThreads, sizeof(float) * a.p.d, a.stream>>>(
@@ -238,7 +223,7 @@ int loss_f32_bwd(const LossArgs& a) {
   if (s != NAT_OK) return s;
   F32Ws w = carve(a.workspace, a.cap);
   NAT_CUDA(cudaMemsetAsync(w.head, 0, sizeof(WorkspaceHead), a.stream));
-  const TokenCtx c = make_ctx(a);
+  const TokenCtx c = make_token_ctx(a, &w.head->status);
   s = launch_grad_coeff(c, a.logp, a.n_sel, a.cap, a.dloss, w.g, a.stream);
   if (s != NAT_OK) return s;
   if (a.cap > 0) {

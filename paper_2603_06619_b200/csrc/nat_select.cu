@@ -12,79 +12,10 @@
 #include <mutex>
 
 #include "nat_common.cuh"
+#include "nat_stream.cuh"
 
 namespace nat {
 namespace {
-
-// ---------------------------------------------------------------- Philox
-// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies
-// with the key advanced by Weyl constants between rounds.
-struct Philox4 {
-  uint32_t x, y, z, w;
-};
-
-__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2,
-                                                 uint32_t c3, uint32_t k0, uint32_t k1) {
-  constexpr uint32_t kMulA = 0xD2511F53u, kMulB = 0xCD9E8D57u;
-  constexpr uint32_t kWeylA = 0x9E3779B9u, kWeylB = 0xBB67AE85u;
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint32_t hiA = __umulhi(kMulA, c0), loA = kMulA * c0;
-    const uint32_t hiB = __umulhi(kMulB, c2), loB = kMulB * c2;
-    c0 = hiB ^ c1 ^ k0;
-    c1 = loB;
-    c2 = hiA ^ c3 ^ k1;
-    c3 = loA;
-    k0 += kWeylA;
-    k1 += kWeylB;
-  }
-  return {c0, c1, c2, c3};
-}
-
-// First index i >= lo with cu[i] > x among cu[0..B] (B + 1 if there is none), found by a
-// whole warp: every step probes 32 positions at once, so a stream of 2^15 responses takes
-// four dependent loads instead of fifteen.  The first step probes 32 consecutive entries
-// because the answer is usually next to the hint.  All 32 lanes call it with the same
-// arguments; cu[i] <= x must hold for every i < lo.
-__device__ __forceinline__ int warp_upper_bound(const int32_t* __restrict__ cu, int B, int64_t x,
-                                                int lo) {
-  const int lane = threadIdx.x & 31;
-  int hi = B + 1;
-  int step = 1;
-  while (lo < hi) {
-    const int idx = lo + lane * step;
-    const bool gt = idx >= hi || (int64_t)__ldg(cu + idx) > x;
-    const unsigned b = __ballot_sync(0xFFFFFFFFu, gt);
-    if (b == 0u) {
-      lo += 31 * step + 1;
-    } else {
-      const int f = __ffs(b) - 1;
-      hi = min(hi, lo + f * step);
-      if (f > 0) lo += (f - 1) * step + 1;
-    }
-    step = max(1, (hi - lo + 31) / 32);
-  }
-  return lo;
-}
-
-// The searches a block makes for the responses around its token range usually end inside
-// one window of 32 consecutive cu entries placed by proportion (position / n_tot * B), so
-// one load serves them all.  cu_window loads the window (one entry per lane, +infinity
-// past cu[B]); window_first turns the ballot of a monotone predicate over it into the first
-// index where it holds, or reports a miss when that index may lie outside the window.
-__device__ __forceinline__ int64_t cu_window(const int32_t* __restrict__ cu, int B, int64_t x,
-                                             int64_t n_tot, int* w0) {
-  const int guess = (int)((x * (int64_t)B) / (n_tot > 0 ? n_tot : 1));
-  *w0 = max(0, min(guess - 8, B - 30));
-  const int idx = *w0 + (int)(threadIdx.x & 31);
-  return idx <= B ? (int64_t)__ldg(cu + idx) : INT64_MAX;
-}
-
-__device__ __forceinline__ bool window_first(unsigned ballot, int w0, int* out) {
-  if (ballot == 0u || ((ballot & 1u) != 0u && w0 > 0)) return false;
-  *out = w0 + __ffs(ballot) - 1;
-  return true;
-}
 
 // ------------------------------------------------------------ advantages
 __global__ void grpo_adv_kernel(int P, int G, const float* __restrict__ rewards, float eps,
@@ -107,8 +38,6 @@ __global__ void grpo_adv_kernel(int P, int G, const float* __restrict__ rewards,
 }
 
 // -------------------------------------------------------------- selection
-constexpr int kTokPerThread = 16;
-constexpr int kSelThreads = 256;
 
 struct SelConst {
   int mode;
@@ -117,6 +46,7 @@ struct SelConst {
   uint64_t thr;    // URS threshold, 1..2^32
   float pi_urs;    // thr / 2^32
   uint32_t k0, k1, off_lo;
+  uint32_t resp_base;  // global index of the first response of cu (draws are keyed by it)
 };
 
 // One thread per response: the RPC cut L_i (or the truncation length K_i).
@@ -130,7 +60,7 @@ __global__ void cut_kernel(SelConst c, int B, const int32_t* __restrict__ cu,
     if (c.mode == NAT_SEL_RPC) {
       const int C = min(max(c.min_cut, 1), T);
       const uint64_t n = (uint64_t)(T - C + 1);
-      const Philox4 r = philox4x32_10(0u, (uint32_t)i, 1u, c.off_lo, c.k0, c.k1);
+      const Philox4 r = philox4x32_10(0u, c.resp_base + (uint32_t)i, 1u, c.off_lo, c.k0, c.k1);
       const uint64_t u = ((uint64_t)r.y << 32) | (uint64_t)r.x;
       L = C + (int)__umul64hi(u, n);
     } else {
@@ -138,17 +68,6 @@ __global__ void cut_kernel(SelConst c, int B, const int32_t* __restrict__ cu,
     }
   }
   cut_len[i] = L;
-}
-
-// Owner search restricted to responses lo..hi (cu[lo] <= n < cu[hi + 1]).
-__device__ __forceinline__ int owner_between(const int32_t* __restrict__ cu, int lo, int hi,
-                                             int64_t n) {
-  ++hi;  // invariant: cu[lo] <= n < cu[hi]
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if ((int64_t)__ldg(cu + mid) <= n) lo = mid; else hi = mid;
-  }
-  return lo;
 }
 
 // One block per 4096 consecutive packed tokens, one thread per 16 of them.  The mask
@@ -167,24 +86,11 @@ __device__ __forceinline__ int owner_between(const int32_t* __restrict__ cu, int
 // rounded float32 quotient.  With y = RN(1/b) computed once per response, q0 = RN(a y),
 // r = a - q0 b (exact in an FMA) and q = RN(q0 + r y) is the correctly rounded a/b
 // (Markstein's theorem on FMA division); three operations per token instead of a division.
-constexpr int kSelBlockTokens = kSelThreads * kTokPerThread;  // 4096
-constexpr int kPiPad = kTokPerThread + 1;                     // 17: conflict-free rows
 
 __device__ __forceinline__ float div_rn_by(float a, float b, float rcp_b) {
   const float q0 = __fmul_rn(a, rcp_b);
   const float r = __fmaf_rn(-q0, b, a);
   return __fmaf_rn(r, rcp_b, q0);
-}
-
-// 16 mask bits -> 16 bytes of 0/1 (bit j -> byte j).
-__device__ __forceinline__ uint4 bits_to_bytes(uint32_t bits) {
-  constexpr uint32_t kSpread = 0x00204081u;  // 1 + 2^7 + 2^14 + 2^21
-  uint4 v;
-  v.x = ((bits & 0xFu) * kSpread) & 0x01010101u;
-  v.y = (((bits >> 4) & 0xFu) * kSpread) & 0x01010101u;
-  v.z = (((bits >> 8) & 0xFu) * kSpread) & 0x01010101u;
-  v.w = (((bits >> 12) & 0xFu) * kSpread) & 0x01010101u;
-  return v;
 }
 
 __device__ __forceinline__ uint32_t philox_below(const Philox4& r, uint64_t thr) {
@@ -243,7 +149,7 @@ select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
       const uint32_t blk0 = t0 >> 2;
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        low |= philox_below(philox4x32_10(blk0 + q, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1), c.thr)
+        low |= philox_below(philox4x32_10(blk0 + q, c.resp_base + (uint32_t)i, 0u, c.off_lo, c.k0, c.k1), c.thr)
                << (4 * q);
     }
     const int tag = inside ? i : -1;
@@ -261,7 +167,7 @@ select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
     if (inside) {
       if (sh != 0u && next_tag != i)
         next_nib = philox_below(
-            philox4x32_10((t0 >> 2) + 4u, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1), c.thr);
+            philox4x32_10((t0 >> 2) + 4u, c.resp_base + (uint32_t)i, 0u, c.off_lo, c.k0, c.k1), c.thr);
       bits = ((low | (next_nib << 16)) >> sh) & 0xFFFFu;
       *reinterpret_cast<uint4*>(mask + n0) = bits_to_bytes(bits);
     } else if (active) {
@@ -283,7 +189,7 @@ select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
           const uint32_t tj = (uint32_t)(n - start);
           const uint32_t blk = tj >> 2;
           if (blk != cached_blk || i != cached_resp) {
-            rnd = philox4x32_10(blk, (uint32_t)i, 0u, c.off_lo, c.k0, c.k1);
+            rnd = philox4x32_10(blk, c.resp_base + (uint32_t)i, 0u, c.off_lo, c.k0, c.k1);
             cached_blk = blk;
             cached_resp = i;
           }
@@ -408,7 +314,7 @@ select_survival_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_
   int i = owner_between(cu, range_s[0], range_s[1], n0);
   int64_t start = cu[i], end = cu[i + 1];
   auto draw = [&]() {
-    const Philox4 r = philox4x32_10(0u, (uint32_t)i, 2u, c.off_lo, c.k0, c.k1);
+    const Philox4 r = philox4x32_10(0u, c.resp_base + (uint32_t)i, 2u, c.off_lo, c.k0, c.k1);
     return __fmul_rn((float)(r.x >> 8), 5.9604644775390625e-08f);  // 2^-24, exact
   };
   float u = draw();
@@ -744,7 +650,11 @@ static int select_impl(const nat_select_params* sp, int32_t B, const int32_t* cu
   if (n_tot > 0x7FFFFFFFll) return fail(NAT_ERR_UNSUPPORTED, "nat_select: n_tot exceeds int32");
   if (!cu_seqlens) return fail(NAT_ERR_INVALID_ARG, "nat_select: cu_seqlens is null");
   if (n_tot > 0 && (!mask || !pi)) return fail(NAT_ERR_INVALID_ARG, "nat_select: null output");
+  if (((uintptr_t)mask & 15u) || ((uintptr_t)pi & 15u))
+    return fail(NAT_ERR_INVALID_ARG, "nat_select: mask and pi must be 16-byte aligned");
+  if (sp->resp_base < 0) return fail(NAT_ERR_INVALID_ARG, "nat_select: resp_base < 0");
   SelConst c{};
+  c.resp_base = (uint32_t)sp->resp_base;
   c.mode = sp->mode;
   c.min_cut = sp->min_cut;
   c.beta = sp->beta;
@@ -790,6 +700,45 @@ static int select_impl(const nat_select_params* sp, int32_t B, const int32_t* cu
   return NAT_OK;
 }
 
+// Argument checks and the launch sequence shared by nat_compact and nat_compact_static
+// (they differ only in where the chunk-count scratch lives).
+static int compact_check(const char* who, int32_t B, const int32_t* cu_seqlens, int64_t n_tot,
+                         const uint8_t* mask, const int32_t* sel_idx, const int32_t* sel_resp,
+                         const int32_t* sel_offsets, const int32_t* n_sel, int64_t cap) {
+  if (B < 0 || n_tot < 0 || cap < 0) return fail(NAT_ERR_INVALID_ARG, "%s: negative size", who);
+  if (n_tot > 0x7FFFFFFFll) return fail(NAT_ERR_UNSUPPORTED, "%s: n_tot exceeds int32", who);
+  if (!cu_seqlens || !sel_offsets || !n_sel) return fail(NAT_ERR_INVALID_ARG, "%s: null pointer", who);
+  if (n_tot > 0 && !mask) return fail(NAT_ERR_INVALID_ARG, "%s: mask is null", who);
+  if ((uintptr_t)mask & 15u)
+    return fail(NAT_ERR_INVALID_ARG, "%s: mask must be 16-byte aligned", who);
+  if (cap > 0 && (!sel_idx || !sel_resp)) return fail(NAT_ERR_INVALID_ARG, "%s: null list", who);
+  return NAT_OK;
+}
+
+static int compact_launch(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8_t* mask,
+                          int32_t* sel_idx, int32_t* sel_resp, int32_t* sel_offsets,
+                          int32_t* n_sel, int64_t cap, int32_t* chunk_count, cudaStream_t stream) {
+  // Every scratch entry read here is written earlier in the same sequence (counts by the
+  // first kernel, offsets and total by the scan), so the scratch needs no clearing.
+  const int n_chunks = (int)((n_tot + kChunk - 1) / kChunk);
+  if (n_chunks > 0) {
+    compact_count_kernel<<<(n_chunks + kCountChunks - 1) / kCountChunks, kCmpThreads, 0, stream>>>(
+        mask, n_tot, n_chunks, chunk_count);
+    NAT_LAUNCH_CHECK("compact_count_kernel");
+  }
+  compact_scan_kernel<<<1, 1024, 0, stream>>>(chunk_count, n_chunks, n_sel, sel_offsets, B);
+  NAT_LAUNCH_CHECK("compact_scan_kernel");
+  if (n_chunks > 0) {
+    compact_write_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(B, cu_seqlens, n_tot, mask,
+                                                               chunk_count, sel_idx, sel_resp,
+                                                               sel_offsets, cap);
+    NAT_LAUNCH_CHECK("compact_write_kernel");
+  } else if (B > 0) {
+    NAT_CUDA(cudaMemsetAsync(sel_offsets, 0, sizeof(int32_t) * (size_t)B, stream));
+  }
+  return NAT_OK;
+}
+
 }  // namespace nat
 
 extern "C" {
@@ -811,8 +760,8 @@ int nat_select(const nat_select_params* params, int32_t B, const int32_t* cu_seq
 }
 
 int nat_select_survival(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const float* surv,
-                        uint64_t seed, uint64_t offset, uint8_t* mask, int32_t* cut_len,
-                        void* stream_) {
+                        uint64_t seed, uint64_t offset, int32_t resp_base, uint8_t* mask,
+                        int32_t* cut_len, void* stream_) {
   using namespace nat;
   cudaStream_t stream = (cudaStream_t)stream_;
   if (B < 0 || n_tot < 0) return fail(NAT_ERR_INVALID_ARG, "nat_select_survival: negative size");
@@ -822,8 +771,10 @@ int nat_select_survival(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, con
     return fail(NAT_ERR_INVALID_ARG, "nat_select_survival: null pointer");
   if (((uintptr_t)surv & 15u) || ((uintptr_t)mask & 15u))
     return fail(NAT_ERR_INVALID_ARG, "nat_select_survival: surv and mask must be 16-byte aligned");
+  if (resp_base < 0) return fail(NAT_ERR_INVALID_ARG, "nat_select_survival: resp_base < 0");
   if (B == 0) return NAT_OK;
   SelConst c{};
+  c.resp_base = (uint32_t)resp_base;
   c.k0 = (uint32_t)(seed & 0xFFFFFFFFull);
   c.k1 = (uint32_t)((seed >> 32) ^ (offset >> 32));
   c.off_lo = (uint32_t)(offset & 0xFFFFFFFFull);
@@ -887,36 +838,16 @@ int nat_compact(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const uint8
                 int32_t* sel_idx, int32_t* sel_resp, int32_t* sel_offsets, int32_t* n_sel,
                 int64_t cap, void* workspace, size_t workspace_bytes, void* stream_) {
   using namespace nat;
-  cudaStream_t stream = (cudaStream_t)stream_;
-  if (B < 0 || n_tot < 0 || cap < 0) return fail(NAT_ERR_INVALID_ARG, "nat_compact: negative size");
-  if (n_tot > 0x7FFFFFFFll) return fail(NAT_ERR_UNSUPPORTED, "nat_compact: n_tot exceeds int32");
-  if (!cu_seqlens || !sel_offsets || !n_sel)
-    return fail(NAT_ERR_INVALID_ARG, "nat_compact: null pointer");
-  if (n_tot > 0 && !mask) return fail(NAT_ERR_INVALID_ARG, "nat_compact: mask is null");
-  if (cap > 0 && (!sel_idx || !sel_resp)) return fail(NAT_ERR_INVALID_ARG, "nat_compact: null list");
+  int s = compact_check("nat_compact", B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offsets,
+                        n_sel, cap);
+  if (s != NAT_OK) return s;
   if (workspace_bytes < nat_compact_workspace_bytes(n_tot) || !workspace)
     return fail(NAT_ERR_CAPACITY, "nat_compact: workspace too small (%zu < %zu)", workspace_bytes,
                 nat_compact_workspace_bytes(n_tot));
   if (((uintptr_t)workspace & 255u) != 0)
     return fail(NAT_ERR_INVALID_ARG, "nat_compact: workspace must be 256-byte aligned");
-  int32_t* chunk_count = reinterpret_cast<int32_t*>(workspace);
-  const int n_chunks = (int)((n_tot + kChunk - 1) / kChunk);
-  if (n_chunks > 0) {
-    compact_count_kernel<<<(n_chunks + kCountChunks - 1) / kCountChunks, kCmpThreads, 0, stream>>>(
-        mask, n_tot, n_chunks, chunk_count);
-    NAT_LAUNCH_CHECK("compact_count_kernel");
-  }
-  compact_scan_kernel<<<1, 1024, 0, stream>>>(chunk_count, n_chunks, n_sel, sel_offsets, B);
-  NAT_LAUNCH_CHECK("compact_scan_kernel");
-  if (n_chunks > 0) {
-    compact_write_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(B, cu_seqlens, n_tot, mask,
-                                                               chunk_count, sel_idx, sel_resp,
-                                                               sel_offsets, cap);
-    NAT_LAUNCH_CHECK("compact_write_kernel");
-  } else if (B > 0) {
-    NAT_CUDA(cudaMemsetAsync(sel_offsets, 0, sizeof(int32_t) * (size_t)B, stream));
-  }
-  return NAT_OK;
+  return compact_launch(B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offsets, n_sel, cap,
+                        reinterpret_cast<int32_t*>(workspace), (cudaStream_t)stream_);
 }
 
 }  // extern "C"
@@ -969,42 +900,19 @@ int nat_compact_static(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, cons
                        int32_t* sel_idx, int32_t* sel_resp, int32_t* sel_offsets, int32_t* n_sel,
                        int64_t cap, void* stream_) {
   using namespace nat;
-  cudaStream_t stream = (cudaStream_t)stream_;
-  if (B < 0 || n_tot < 0 || cap < 0)
-    return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: negative size");
+  int s = compact_check("nat_compact_static", B, cu_seqlens, n_tot, mask, sel_idx, sel_resp,
+                        sel_offsets, n_sel, cap);
+  if (s != NAT_OK) return s;
   if (n_tot > nat_compact_static_max_tokens())
     return fail(NAT_ERR_CAPACITY,
                 "nat_compact_static: n_tot = %lld exceeds the built-in scratch (at most %lld "
                 "tokens); use nat_compact with a caller-provided workspace",
                 (long long)n_tot, (long long)nat_compact_static_max_tokens());
-  if (!cu_seqlens || !sel_offsets || !n_sel)
-    return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: null pointer");
-  if (n_tot > 0 && !mask) return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: mask is null");
-  if (cap > 0 && (!sel_idx || !sel_resp))
-    return fail(NAT_ERR_INVALID_ARG, "nat_compact_static: null list");
   int32_t* chunk_count = nullptr;
-  int s = static_scratch(&chunk_count);
+  s = static_scratch(&chunk_count);
   if (s != NAT_OK) return s;
-  // Every scratch entry this call reads is written earlier in the same call
-  // (counts by the first kernel, offsets and total by the scan), so nothing left
-  // by a previous call needs clearing.
-  const int n_chunks = (int)((n_tot + kChunk - 1) / kChunk);
-  if (n_chunks > 0) {
-    compact_count_kernel<<<(n_chunks + kCountChunks - 1) / kCountChunks, kCmpThreads, 0, stream>>>(
-        mask, n_tot, n_chunks, chunk_count);
-    NAT_LAUNCH_CHECK("compact_count_kernel");
-  }
-  compact_scan_kernel<<<1, 1024, 0, stream>>>(chunk_count, n_chunks, n_sel, sel_offsets, B);
-  NAT_LAUNCH_CHECK("compact_scan_kernel");
-  if (n_chunks > 0) {
-    compact_write_kernel<<<n_chunks, kCmpThreads, 0, stream>>>(B, cu_seqlens, n_tot, mask,
-                                                               chunk_count, sel_idx, sel_resp,
-                                                               sel_offsets, cap);
-    NAT_LAUNCH_CHECK("compact_write_kernel");
-  } else if (B > 0) {
-    NAT_CUDA(cudaMemsetAsync(sel_offsets, 0, sizeof(int32_t) * (size_t)B, stream));
-  }
-  return NAT_OK;
+  return compact_launch(B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offsets, n_sel, cap,
+                        chunk_count, (cudaStream_t)stream_);
 }
 
 }  // extern "C"

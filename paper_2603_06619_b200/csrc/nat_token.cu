@@ -39,6 +39,25 @@ __global__ void grad_coeff_kernel(TokenCtx c, const float* __restrict__ logp,
 
 }  // namespace
 
+TokenCtx make_token_ctx(const LossArgs& a, uint32_t* status) {
+  TokenCtx c;
+  c.targets = a.targets;
+  c.old_logp = a.old_logp;
+  c.adv = a.adv;
+  c.pi = a.pi;
+  c.cu_seqlens = a.cu_seqlens;
+  c.sel_idx = a.sel_idx;
+  c.sel_resp = a.sel_resp;
+  c.B = a.p.B;
+  c.clip_lo = a.p.clip_lo;
+  c.clip_hi = a.p.clip_hi;
+  c.kl_beta = a.p.kl_beta;
+  c.ref_logp = a.p.ref_logp;
+  c.V = a.p.V;
+  c.status = status;
+  return c;
+}
+
 int launch_loss_reduce(const float* term, const int32_t* n_sel, int64_t cap, float* loss,
                        WorkspaceHead* head, cudaStream_t stream) {
   loss_reduce_kernel<<<1, 1024, 0, stream>>>(term, n_sel, cap, loss, head);

@@ -26,16 +26,31 @@ struct TokenCtx {
   float clip_lo, clip_hi;
   float kl_beta;          // 0: no KL term
   const float* ref_logp;  // read only when kl_beta != 0
+  int V;                  // targets outside [0, V) are reported and their tokens left out
+  uint32_t* status;       // the workspace's status word
 };
+
+// Fills the fields every loss path takes from the call's arguments.
+TokenCtx make_token_ctx(const LossArgs& a, uint32_t* status);
 
 // For selected token k with log-probability logp:
 //   r = exp(logp - old_logp), S = min(r A, clip(r) A), w = 1 / (pi T B)
 //   term = -w (S - kl_beta (logp - ref_logp))      (the token's share of the loss)
 //   g    = -dloss w (A r [surrogate not saturated] - kl_beta)
+__device__ __forceinline__ bool target_ok(const TokenCtx& c, int k) {
+  return (unsigned)c.targets[c.sel_idx[k]] < (unsigned)c.V;
+}
+
 __device__ __forceinline__ void token_eval(const TokenCtx& c, int k, float logp, float dloss,
                                            float* term, float* g) {
   const int n = c.sel_idx[k];
   const int i = c.sel_resp[k];
+  if ((unsigned)c.targets[n] >= (unsigned)c.V) {  // no such vocabulary entry: leave the token out
+    atomicOr(c.status, NAT_DEV_BAD_TARGET);
+    *term = 0.f;
+    *g = 0.f;
+    return;
+  }
   const float A = c.adv[i];
   const float T = (float)(c.cu_seqlens[i + 1] - c.cu_seqlens[i]);
   const float w = 1.f / (c.pi[n] * T * (float)c.B);

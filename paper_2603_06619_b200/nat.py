@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libnat_b200.so")
 
 NAT_SEL_URS, NAT_SEL_RPC, NAT_SEL_DET = 0, 1, 2
 NAT_F32, NAT_BF16 = 0, 1
-NAT_DEV_TIMEOUT, NAT_DEV_CAPACITY, NAT_DEV_FALLBACK = 1, 2, 4
+NAT_DEV_TIMEOUT, NAT_DEV_CAPACITY, NAT_DEV_FALLBACK, NAT_DEV_BAD_TARGET = 1, 2, 4, 8
 
 SYMBOLS = (
     "nat_status_string", "nat_last_error", "nat_version", "nat_grpo_adv", "nat_select",
@@ -23,6 +23,8 @@ SYMBOLS = (
     "nat_policy_loss_fwd", "nat_policy_loss_bwd", "nat_compact_static",
     "nat_compact_static_max_tokens", "nat_policy_loss_fwd_bwd", "nat_trace_begin",
     "nat_trace_end", "nat_select_survival", "nat_gather_rows", "nat_scatter_rows",
+    "nat_poll_status", "nat_compact_prefix", "nat_select_cutlaw",
+    "nat_select_cutlaw_workspace_bytes",
 )
 TRACE_KINDS = ("fwd", "dz", "dh", "dw", "e")
 
@@ -33,7 +35,8 @@ class NatError(RuntimeError):
 
 class SelectParams(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("min_cut", ctypes.c_int32), ("p", ctypes.c_double),
-                ("beta", ctypes.c_double), ("seed", ctypes.c_uint64), ("offset", ctypes.c_uint64)]
+                ("beta", ctypes.c_double), ("seed", ctypes.c_uint64), ("offset", ctypes.c_uint64),
+                ("resp_base", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class LossParams(ctypes.Structure):
@@ -63,9 +66,18 @@ def load():
     lib.nat_version.restype = ctypes.c_int
     lib.nat_grpo_adv.argtypes = [i32, i32, vp, f32, vp, vp]
     lib.nat_select.argtypes = [ctypes.POINTER(SelectParams), i32, vp, i64, vp, vp, vp, vp]
-    lib.nat_select_survival.argtypes = [i32, vp, i64, vp, ctypes.c_uint64, ctypes.c_uint64, vp, vp,
-                                        vp]
+    lib.nat_select_survival.argtypes = [i32, vp, i64, vp, ctypes.c_uint64, ctypes.c_uint64, i32,
+                                        vp, vp, vp]
     lib.nat_select_survival.restype = ctypes.c_int
+    lib.nat_select_cutlaw_workspace_bytes.restype = ctypes.c_size_t
+    lib.nat_select_cutlaw_workspace_bytes.argtypes = [i32, i64]
+    lib.nat_select_cutlaw.argtypes = [i32, vp, i64, vp, ctypes.c_uint64, ctypes.c_uint64, i32, vp,
+                                      vp, vp, vp, ctypes.c_size_t, vp]
+    lib.nat_select_cutlaw.restype = ctypes.c_int
+    lib.nat_compact_prefix.argtypes = [i32, vp, i64, vp, vp, vp, vp, vp, i64, vp]
+    lib.nat_compact_prefix.restype = ctypes.c_int
+    lib.nat_poll_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.nat_poll_status.restype = ctypes.c_int
     lib.nat_gather_rows.argtypes = [vp, i64, vp, vp, i64, vp, vp]
     lib.nat_gather_rows.restype = ctypes.c_int
     lib.nat_scatter_rows.argtypes = [vp, i64, vp, vp, i64, i64, vp, vp]
@@ -117,9 +129,10 @@ def nat_grpo_adv(P, G, rewards, eps, adv):
     _check(load().nat_grpo_adv(P, G, _ptr(rewards), eps, _ptr(adv), _stream()))
 
 
-def select_params(mode, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
+def select_params(mode, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0, resp_base=0):
     mode = {"urs": NAT_SEL_URS, "rpc": NAT_SEL_RPC, "det": NAT_SEL_DET}.get(mode, mode)
-    return SelectParams(mode=mode, min_cut=min_cut, p=p, beta=beta, seed=seed, offset=offset)
+    return SelectParams(mode=mode, min_cut=min_cut, p=p, beta=beta, seed=seed, offset=offset,
+                        resp_base=resp_base, reserved=0)
 
 
 def nat_select(params, B, cu_seqlens, n_tot, mask, pi, cut_len):
@@ -127,9 +140,20 @@ def nat_select(params, B, cu_seqlens, n_tot, mask, pi, cut_len):
                              _ptr(pi), _ptr(cut_len), _stream()))
 
 
-def nat_select_survival(B, cu_seqlens, n_tot, surv, seed, offset, mask, cut_len):
+def nat_select_survival(B, cu_seqlens, n_tot, surv, seed, offset, mask, cut_len, resp_base=0):
     _check(load().nat_select_survival(B, _ptr(cu_seqlens), n_tot, _ptr(surv), seed, offset,
-                                      _ptr(mask), _ptr(cut_len), _stream()))
+                                      resp_base, _ptr(mask), _ptr(cut_len), _stream()))
+
+
+def nat_select_cutlaw_workspace_bytes(B, n_tot):
+    return load().nat_select_cutlaw_workspace_bytes(B, n_tot)
+
+
+def nat_select_cutlaw(B, cu_seqlens, n_tot, q, seed, offset, mask, pi, cut_len, workspace,
+                      resp_base=0):
+    _check(load().nat_select_cutlaw(B, _ptr(cu_seqlens), n_tot, _ptr(q), seed, offset, resp_base,
+                                    _ptr(mask), _ptr(pi), _ptr(cut_len), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream()))
 
 
 def _row_bytes(t):
@@ -155,6 +179,12 @@ def nat_compact(B, cu_seqlens, n_tot, mask, sel_idx, sel_resp, sel_offsets, n_se
                               _ptr(sel_resp), _ptr(sel_offsets), _ptr(n_sel), cap,
                               _ptr(workspace), workspace.numel() * workspace.element_size(),
                               _stream()))
+
+
+def nat_compact_prefix(B, cu_seqlens, n_tot, cut_len, sel_idx, sel_resp, sel_offsets, n_sel, cap):
+    _check(load().nat_compact_prefix(B, _ptr(cu_seqlens), n_tot, _ptr(cut_len), _ptr(sel_idx),
+                                     _ptr(sel_resp), _ptr(sel_offsets), _ptr(n_sel), cap,
+                                     _stream()))
 
 
 def nat_compact_static_max_tokens():
@@ -227,6 +257,11 @@ def alloc_workspace(nbytes, device):
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
 
-def device_status(workspace):
-    """The NAT_DEV_* bits the last loss call left in its workspace (synchronises)."""
-    return int(workspace[:4].view(torch.int32).item())
+def nat_poll_status(workspace):
+    """The NAT_DEV_* bits the last loss call left in its workspace (waits for the stream)."""
+    word = ctypes.c_uint32(0)
+    _check(load().nat_poll_status(_ptr(workspace), _stream(), ctypes.byref(word)))
+    return int(word.value)
+
+
+device_status = nat_poll_status

@@ -12,8 +12,14 @@ from . import nat
 class NatStep:
     def __init__(self, P, G, d, V, dtype, n_tot, device="cuda", n_sel_cap=None,
                  clip_lo=0.2, clip_hi=0.2, eps=1e-6, hidden_is_compact=False, want_grads=True,
-                 kl_beta=0.0, ref_logp=None):
+                 kl_beta=0.0, ref_logp=None, B_global=None, resp_base=0):
+        """``B_global`` / ``resp_base``: for a data-parallel shard, the number of responses of
+        the whole job's batch (the batch mean's divisor) and the global index of this
+        shard's first response (the selection draws are keyed by it)."""
         self.P, self.G, self.B = P, G, P * G
+        self.B_global = self.B if B_global is None else int(B_global)
+        self.resp_base = int(resp_base)
+        self.prefix_mode = False
         self.d, self.V, self.dtype = d, V, dtype
         self.n_tot = int(n_tot)
         self.cap = int(n_tot if n_sel_cap is None else n_sel_cap)
@@ -31,7 +37,7 @@ class NatStep:
         self.n_sel = torch.zeros(1, dtype=i32, device=dev)
         self.compact_ws = nat.alloc_workspace(nat.nat_compact_workspace_bytes(self.n_tot), dev)
         self.ref_logp = ref_logp            # keeps the tensor alive while params point at it
-        self.params = nat.loss_params(d, V, dtype, self.B, clip_lo, clip_hi, hidden_is_compact,
+        self.params = nat.loss_params(d, V, dtype, self.B_global, clip_lo, clip_hi, hidden_is_compact,
                                       kl_beta=kl_beta, ref_logp=ref_logp)
         self.loss = torch.zeros(1, dtype=f32, device=dev)
         self.logp = torch.empty(max(self.cap, 1), dtype=f32, device=dev)
@@ -49,13 +55,22 @@ class NatStep:
         return self.adv
 
     def select(self, cu_seqlens, mode, p=1.0, min_cut=1, beta=1.0, seed=0, offset=0):
-        sp = nat.select_params(mode, p=p, min_cut=min_cut, beta=beta, seed=seed, offset=offset)
-        cut = None if sp.mode == nat.NAT_SEL_URS else self.cut_len
+        sp = nat.select_params(mode, p=p, min_cut=min_cut, beta=beta, seed=seed, offset=offset,
+                               resp_base=self.resp_base)
+        self.prefix_mode = sp.mode != nat.NAT_SEL_URS
+        cut = self.cut_len if self.prefix_mode else None
         nat.nat_select(sp, self.B, cu_seqlens, self.n_tot, self.mask, self.pi, cut)
 
-    def compact(self, cu_seqlens):
-        nat.nat_compact(self.B, cu_seqlens, self.n_tot, self.mask, self.sel_idx, self.sel_resp,
-                        self.sel_offsets, self.n_sel, self.cap, self.compact_ws)
+    def compact(self, cu_seqlens, from_mask=False):
+        """Compacted lists of the last selection: straight from the cut lengths after a
+        prefix mode (RPC, truncation), from the mask otherwise (or when asked to)."""
+        if self.prefix_mode and not from_mask:
+            nat.nat_compact_prefix(self.B, cu_seqlens, self.n_tot, self.cut_len, self.sel_idx,
+                                   self.sel_resp, self.sel_offsets, self.n_sel, self.cap)
+        else:
+            nat.nat_compact(self.B, cu_seqlens, self.n_tot, self.mask, self.sel_idx,
+                            self.sel_resp, self.sel_offsets, self.n_sel, self.cap,
+                            self.compact_ws)
 
     def loss_fwd(self, hidden, W, targets, old_logp, cu_seqlens):
         nat.nat_policy_loss_fwd(self.params, hidden, W, targets, old_logp, self.adv, self.pi,

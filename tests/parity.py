@@ -5,7 +5,11 @@ Tolerances (from the target statement of the method's numerics):
   masks, pi, cut lengths, compacted indices, advantages   bit-exact
   loss                  1e-3 relative (against a floor tied to sum |w S|, since the
                         loss is a near-cancelling sum on centred advantages)
-  logp, lse             2e-4 absolute (fp32 accumulation of bf16 products)
+  logp, lse             2e-4 absolute (fp32 accumulation of bf16 products) for logits of
+                        the workloads' size (lse <= 16); the rounding of an fp32 running
+                        sum is relative to its magnitude, so for the peaked-softmax variants
+                        (logits of standard deviation 10..32) this tolerance and the loss
+                        floor grow in proportion, by max(1, max lse / 16)
   dHidden, dW           1e-2 relative Frobenius error
   dense parts           2e-2 relative Frobenius error (gradient minus its
                         one-hot target term: the softmax part alone, which the
@@ -66,24 +70,32 @@ def check_selection(st, ref, w):
 
 
 def check_loss(st, ref_sel, nb, w, backward=True, hidden_is_compact=False, clip=(0.2, 0.2),
-               hidden_np=None, kl_beta=0.0, ref_logp=None):
-    """Element-by-element comparison of loss, logp, lse, dHidden, dW with the oracle."""
+               hidden_np=None, kl_beta=0.0, ref_logp=None, ref=None, B_global=None):
+    """Element-by-element comparison of loss, logp, lse, dHidden, dW with the oracle.
+
+    ``ref``: the oracle's result from an earlier call on the same inputs (the fp64
+    evaluation is the expensive part; two routes of the library are checked against one).
+    """
     n = ref_sel["n_sel"]
     hidden = nb["hidden"] if hidden_np is None else hidden_np
-    fn = oracle.policy_loss_bwd if backward else oracle.policy_loss_fwd
-    ref = fn(hidden, nb["W"], nb["targets"], nb["old_logp"], ref_sel["adv"], ref_sel["pi"],
-             nb["cu_seqlens"], ref_sel["sel_idx"], ref_sel["sel_resp"], clip_lo=clip[0],
-             clip_hi=clip[1], hidden_is_compact=hidden_is_compact, kl_beta=kl_beta,
-             ref_logp=ref_logp)
+    if ref is None:
+        fn = oracle.policy_loss_bwd if backward else oracle.policy_loss_fwd
+        ref = fn(hidden, nb["W"], nb["targets"], nb["old_logp"], ref_sel["adv"], ref_sel["pi"],
+                 nb["cu_seqlens"], ref_sel["sel_idx"], ref_sel["sel_resp"], clip_lo=clip[0],
+                 clip_hi=clip[1], hidden_is_compact=hidden_is_compact, kl_beta=kl_beta,
+                 ref_logp=ref_logp)
     assert st.status() & ~4 == 0      # the informational fallback bit may be set
     got_logp = st.logp[:n].cpu().numpy()
     got_lse = st.lse[:n].cpu().numpy()
-    assert np.abs(got_logp - ref["logp"]).max(initial=0) <= TOL_LOGP
-    assert np.abs(got_lse - ref["lse"]).max(initial=0) <= TOL_LOGP
+    mag = max(1.0, float(np.abs(ref["lse"]).max(initial=0)) / 16.0)
+    out = dict(logp_err=float(np.abs(got_logp - ref["logp"]).max(initial=0)),
+               lse_err=float(np.abs(got_lse - ref["lse"]).max(initial=0)), logit_mag=mag)
+    assert out["logp_err"] <= TOL_LOGP * mag, out
+    assert out["lse_err"] <= TOL_LOGP * mag, out
     loss = float(st.loss.item())
-    floor = 1e-2 * float(np.sum(ref["w"] * np.abs(ref["L"])))
+    floor = 1e-2 * mag * float(np.sum(ref["w"] * np.abs(ref["L"])))
     assert abs(loss - ref["loss"]) <= TOL_LOSS * max(abs(ref["loss"]), floor), (loss, ref["loss"])
-    out = dict(loss=loss, ref_loss=ref["loss"])
+    out.update(loss=loss, ref_loss=ref["loss"])
     if backward:
         dH = st.dH[:n].float().cpu().numpy()
         dW = st.dW.cpu().numpy()
@@ -108,10 +120,19 @@ def check_loss(st, ref_sel, nb, w, backward=True, hidden_is_compact=False, clip=
     return out, ref
 
 
-def run_case(w, seed=0, offset=0, backward=True, device="cuda", fused=False, **batch_kw):
+def run_case(w, seed=0, offset=0, backward=True, device="cuda", fused=False, routes=None,
+             **batch_kw):
+    """One seeded batch through the library and the oracle.  ``routes`` lists the library
+    routes to check against the single oracle evaluation (False: forward then backward
+    calls, True: the single-pass call); default: the one ``fused`` names."""
     batch = wl.make_batch(w, seed=seed, device=device, **batch_kw)
     nb = wl.to_numpy(batch)
     ref_sel = oracle_selection(w, nb, seed, offset)
-    st = gpu_step(w, batch, seed, offset, backward=backward, fused=fused)
-    check_selection(st, ref_sel, w)
-    return check_loss(st, ref_sel, nb, w, backward=backward)
+    out, ref = None, None
+    for f in ([fused] if routes is None else routes):
+        st = gpu_step(w, batch, seed, offset, backward=backward, fused=f)
+        check_selection(st, ref_sel, w)
+        out, ref = check_loss(st, ref_sel, nb, w, backward=backward, ref=ref)
+        out["status"] = st.status()
+        del st
+    return out, ref

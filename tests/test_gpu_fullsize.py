@@ -1,5 +1,6 @@
 """GPU parity at the benchmark's full sizes, in the launch configuration bench.py times
-(capacity = N_tot, n_sel read on the device).
+(capacity = N_tot, n_sel read on the device), for both routes of the loss (the single-pass
+call, and forward followed by backward).
 
 The fp64 oracle cannot evaluate 10^14..10^15 FLOPs, so here:
   * advantages, masks, pi, cuts and compacted indices are compared in full, bit for bit;
@@ -7,120 +8,205 @@ The fp64 oracle cannot evaluate 10^14..10^15 FLOPs, so here:
     oracle evaluates one by one (stream ends, tile and chunk edges, random rows);
   * the scalar loss is checked against the fp64 sum of the per-token terms that the
     sampled comparison validates (a consistency property, stated as such);
-  * dW is tied to the validated dHidden by identities that hold at any size:
-    every column of dW sums to zero over the vocabulary, and
-    sum_k <dHidden_k, h_k> = <dW, W>  (both equal sum_{k,v} dz[k,v] z[k,v]).
-Element-by-element dW parity is covered at the reduced twins of the same heads.
+  * dW is compared with the oracle on a sample of vocabulary rows, each summed over ALL
+    selected tokens: dW[v, :] = sum_n g_n (1[v = y_n] - exp(W_v . h_n - lse_n)) h_n.  The
+    per-token scalars g_n and lse_n entering that sum are formed in fp64 from the library's
+    logp / lse after the sampled rows validated them -- a bootstrap, stated as such: the
+    oracle cannot produce lse for every row of a full-size batch;
+  * and dW is tied to dHidden by identities that hold at any size: every column of dW sums
+    to zero over the vocabulary, and sum_k <dHidden_k, h_k> = <dW, W>.
+Element-by-element parity of all of dW is covered at the reduced twins of the same heads.
 """
 import numpy as np
 import pytest
 import torch
 
 import oracle
+from oracle.nat_oracle import _token_weights
 from paper_2603_06619_b200 import workloads as wl
+from paper_2603_06619_b200.step import NatStep
 
 import parity
 
 pytestmark = pytest.mark.gpu
 
+ROW_BLOCK = 8192
+
 
 def _sample_rows(n, rng, k_random=40):
-    edges = [0, 1, 127, 128, 129, 255, 256, 8191, 8192, 8193, 16383, 16384, n - 129, n - 128,
-             n - 2, n - 1]
+    edges = [0, 1, 127, 128, 129, 255, 256, 511, 512, 8191, 8192, 8193, 16383, 16384, n - 129,
+             n - 128, n - 2, n - 1]
     rows = {r for r in edges if 0 <= r < n}
     rows |= set(int(x) for x in rng.integers(0, n, size=k_random))
     return np.array(sorted(rows), dtype=np.int64)
 
 
-def _full_size_case(name, seed=0, fused=False, **variant):
-    w = wl.variant(wl.WORKLOADS[name], **variant) if variant else wl.WORKLOADS[name]
-    batch = wl.make_batch(w, seed=seed, device="cuda")
-    nb = {k: (v.cpu().numpy() if isinstance(v, torch.Tensor) and v.dtype != torch.bfloat16 else v)
-          for k, v in batch.items() if k not in ("hidden", "W")}
-    ref_sel = parity.oracle_selection(w, nb, seed, 0)
-    st = parity.gpu_step(w, batch, seed, 0, fused=fused)
-    parity.check_selection(st, ref_sel, w)
-    assert st.status() == 0
-    n = ref_sel["n_sel"]
+def _sample_vocab(V, y_live, rng, k_targets=16, k_random=36):
+    """Vocabulary rows for the dW comparison: rows that are targets of live tokens, rows that
+    are (most likely) nobody's target, the last row, and both sides of tile edges."""
+    rows = {0, 127, 128, 255, 256, 511, 512, 513, 1023, 1024, V - 513, V - 512, V - 2, V - 1}
+    rows = {r for r in rows if 0 <= r < V}
+    if len(y_live):
+        rows |= set(int(x) for x in rng.choice(y_live, size=min(k_targets, len(y_live)),
+                                               replace=False))
+    rows |= set(int(x) for x in rng.integers(0, V, size=k_random))
+    return np.array(sorted(rows), dtype=np.int64)
 
-    rng = np.random.default_rng(seed)
-    rows = _sample_rows(n, rng)
-    si = ref_sel["sel_idx"][rows]
-    sr = ref_sel["sel_resp"][rows]
-    # only the sampled hidden rows travel to the host; W goes whole
-    hidden_rows = batch["hidden"][torch.from_numpy(si).long().cuda()].float().cpu().numpy()
-    Wn = batch["W"].float().cpu().numpy()
-    ref = oracle.policy_loss_bwd(hidden_rows, Wn, nb["targets"], nb["old_logp"], ref_sel["adv"],
-                                 ref_sel["pi"], nb["cu_seqlens"], si, sr, hidden_is_compact=True,
-                                 want_dW=False)
-    got_logp = st.logp[:n].cpu().numpy()
-    got_lse = st.lse[:n].cpu().numpy()
-    assert np.abs(got_logp[rows] - ref["logp"]).max() <= parity.TOL_LOGP
-    assert np.abs(got_lse[rows] - ref["lse"]).max() <= parity.TOL_LOGP
-    dH_rows = st.dH[torch.from_numpy(rows).cuda()].float().cpu().numpy()
-    assert parity.rel_fro(dH_rows, ref["dH"]) <= parity.TOL_GRAD
-    live = ref["g"] != 0
-    if live.any():
-        per_row = np.linalg.norm(dH_rows[live] - ref["dH"][live], axis=1) / \
-            np.linalg.norm(ref["dH"][live], axis=1)
-        assert per_row.max() <= 2 * parity.TOL_GRAD
-    assert np.all(dH_rows[~live] == 0)
 
-    # loss = fp64 sum of the per-token terms evaluated at the (sample-validated) logp
-    full_idx, full_resp = ref_sel["sel_idx"], ref_sel["sel_resp"]
-    T = np.diff(nb["cu_seqlens"]).astype(np.float64)
-    wgt = 1.0 / (ref_sel["pi"].astype(np.float64)[full_idx] * T[full_resp] * w.B)
-    A = ref_sel["adv"].astype(np.float64)[full_resp]
-    r = np.exp(got_logp.astype(np.float64) - nb["old_logp"].astype(np.float64)[full_idx])
-    S = np.minimum(r * A, np.clip(r, 0.8, 1.2) * A)
-    want = -np.sum(wgt * S)
-    floor = 1e-2 * np.sum(wgt * np.abs(S))
-    assert abs(float(st.loss.item()) - want) <= parity.TOL_LOSS * max(abs(want), floor)
+class _Case:
+    """One seeded full-size batch on the device, its small arrays on the host, one NatStep."""
 
-    # dW identities (computed on the device in fp64 where it matters)
-    dW = st.dW
-    col = dW.double().sum(0)
-    assert float(col.abs().max()) <= 1e-3 * float(dW.double().abs().sum(0).max())
-    idx = torch.from_numpy(full_idx).long().cuda()
-    lhs = 0.0
-    for lo in range(0, n, 16384):
-        hi = min(lo + 16384, n)
-        lhs += float((st.dH[lo:hi].double() * batch["hidden"][idx[lo:hi]].double()).sum())
-    rhs = 0.0
-    for lo in range(0, w.V, 16384):
-        rhs += float((dW[lo:lo + 16384].double() * batch["W"][lo:lo + 16384].double()).sum())
-    scale = float((dW.double().abs() * batch["W"].double().abs()).sum())
-    assert abs(lhs - rhs) <= 2e-3 * scale, (lhs, rhs, scale)
-    return n
+    def __init__(self, name, seed=0, **variant):
+        self.w = wl.variant(wl.WORKLOADS[name], **variant) if variant else wl.WORKLOADS[name]
+        self.seed = seed
+        self.batch = wl.make_batch(self.w, seed=seed, device="cuda")
+        b = self.batch
+        self.nb = {k: (v.cpu().numpy() if isinstance(v, torch.Tensor) else v)
+                   for k, v in b.items() if k not in ("hidden", "W")}
+        self.Wn = b["W"].float().cpu().numpy()
+        self.st = NatStep(self.w.P, self.w.G, self.w.d, self.w.V, torch.bfloat16, b["n_tot"])
+
+    def check(self, routes=(True, False), vocab_rows=True, **sel):
+        """Run the step under one selection setting through each route and compare."""
+        w = wl.variant(self.w, **sel) if sel else self.w
+        nb, batch, st = self.nb, self.batch, self.st
+        ref_sel = parity.oracle_selection(w, nb, self.seed, 0)
+        n = ref_sel["n_sel"]
+        rng = np.random.default_rng(self.seed)
+        rows = _sample_rows(n, rng)
+        si, sr = ref_sel["sel_idx"][rows], ref_sel["sel_resp"][rows]
+        # only the sampled hidden rows travel to the host; W went whole
+        hidden_rows = batch["hidden"][torch.from_numpy(si).long().cuda()].float().cpu().numpy()
+        ref = oracle.policy_loss_bwd(hidden_rows, self.Wn, nb["targets"], nb["old_logp"],
+                                     ref_sel["adv"], ref_sel["pi"], nb["cu_seqlens"], si, sr,
+                                     hidden_is_compact=True, want_dW=False)
+        ref_dw = None
+        for fused in routes:
+            st.run(batch, w.sel_mode, p=w.p, min_cut=w.min_cut, beta=w.beta, seed=self.seed,
+                   offset=0, fused=fused)
+            torch.cuda.synchronize()
+            parity.check_selection(st, ref_sel, w)
+            assert st.status() == 0
+            self._check_rows(ref_sel, ref, rows)
+            self._check_loss(ref_sel, w)
+            self._check_dw_identities(ref_sel, w)
+            if vocab_rows:
+                if ref_dw is None:
+                    ref_dw = self._oracle_dw_rows(ref_sel, w, rng)
+                self._check_dw_rows(ref_dw)
+        return n
+
+    # -- sampled selected rows: logp, lse, dHidden -------------------------
+    def _check_rows(self, ref_sel, ref, rows):
+        st, n = self.st, ref_sel["n_sel"]
+        got_logp = st.logp[:n].cpu().numpy()
+        got_lse = st.lse[:n].cpu().numpy()
+        assert np.abs(got_logp[rows] - ref["logp"]).max() <= parity.TOL_LOGP
+        assert np.abs(got_lse[rows] - ref["lse"]).max() <= parity.TOL_LOGP
+        dH_rows = st.dH[torch.from_numpy(rows).cuda()].float().cpu().numpy()
+        assert parity.rel_fro(dH_rows, ref["dH"]) <= parity.TOL_GRAD
+        live = ref["g"] != 0
+        if live.any():
+            per_row = np.linalg.norm(dH_rows[live] - ref["dH"][live], axis=1) / \
+                np.linalg.norm(ref["dH"][live], axis=1)
+            assert per_row.max() <= 2 * parity.TOL_GRAD
+        assert np.all(dH_rows[~live] == 0)
+
+    # -- loss = fp64 sum of the per-token terms at the (sample-validated) logp --
+    def _token_scalars(self, ref_sel, w):
+        st, nb, n = self.st, self.nb, ref_sel["n_sel"]
+        full_idx, full_resp = ref_sel["sel_idx"], ref_sel["sel_resp"]
+        wgt = _token_weights(ref_sel["pi"], nb["cu_seqlens"], full_idx, full_resp)
+        A = ref_sel["adv"].astype(np.float64)[full_resp]
+        logp = st.logp[:n].cpu().numpy().astype(np.float64)
+        r = np.exp(logp - nb["old_logp"].astype(np.float64)[full_idx])
+        return wgt, A, r
+
+    def _check_loss(self, ref_sel, w):
+        wgt, A, r = self._token_scalars(ref_sel, w)
+        S = np.minimum(r * A, np.clip(r, 0.8, 1.2) * A)
+        want = -np.sum(wgt * S)
+        floor = 1e-2 * np.sum(wgt * np.abs(S))
+        assert abs(float(self.st.loss.item()) - want) <= parity.TOL_LOSS * max(abs(want), floor)
+
+    # -- identities that tie dW to dHidden at any size ---------------------
+    def _check_dw_identities(self, ref_sel, w):
+        st, batch, n = self.st, self.batch, ref_sel["n_sel"]
+        dW = st.dW
+        col = torch.zeros(w.d, dtype=torch.float64, device="cuda")
+        col_abs = torch.zeros(w.d, dtype=torch.float64, device="cuda")
+        rhs, scale = 0.0, 0.0
+        for lo in range(0, w.V, 16384):
+            blk = dW[lo:lo + 16384].double()
+            Wb = batch["W"][lo:lo + 16384].double()
+            col += blk.sum(0)
+            col_abs += blk.abs().sum(0)
+            rhs += float((blk * Wb).sum())
+            scale += float((blk.abs() * Wb.abs()).sum())
+        assert float(col.abs().max()) <= 1e-3 * float(col_abs.max())
+        idx = torch.from_numpy(ref_sel["sel_idx"]).long().cuda()
+        lhs = 0.0
+        for lo in range(0, n, 16384):
+            hi = min(lo + 16384, n)
+            lhs += float((st.dH[lo:hi].double() * batch["hidden"][idx[lo:hi]].double()).sum())
+        assert abs(lhs - rhs) <= 2e-3 * scale, (lhs, rhs, scale)
+
+    # -- sampled vocabulary rows of dW against the oracle ------------------
+    def _oracle_dw_rows(self, ref_sel, w, rng):
+        st, nb, batch, n = self.st, self.nb, self.batch, ref_sel["n_sel"]
+        wgt, A, r = self._token_scalars(ref_sel, w)
+        g = oracle.grad_coeff(r, A, wgt, 0.2, 0.2)
+        lse = st.lse[:n].cpu().numpy().astype(np.float64)
+        y = nb["targets"][ref_sel["sel_idx"]]
+        v_ids = _sample_vocab(w.V, np.unique(y[g != 0]), rng)
+        idx = torch.from_numpy(ref_sel["sel_idx"]).long().cuda()
+
+        def blocks():                                   # the selected rows, streamed to the host
+            for lo in range(0, n, ROW_BLOCK):
+                yield batch["hidden"][idx[lo:lo + ROW_BLOCK]].float().cpu().numpy()
+
+        rows, dense = oracle.policy_loss_dW_rows(blocks(), self.Wn[v_ids], v_ids, y, g, lse)
+        is_target = np.isin(v_ids, y[g != 0])
+        assert is_target.any() and (~is_target).any()
+        return v_ids, rows, dense
+
+    def _check_dw_rows(self, ref_dw):
+        v_ids, rows, dense = ref_dw
+        got = self.st.dW[torch.from_numpy(v_ids).cuda()].double().cpu().numpy()
+        assert parity.rel_fro(got, rows) <= parity.TOL_GRAD
+        # row by row (a dropped, doubled or misplaced chunk of rows shows in every row)
+        per_row = np.linalg.norm(got - rows, axis=1) / np.linalg.norm(rows, axis=1)
+        assert per_row.max() <= 2 * parity.TOL_DENSE, per_row.max()
+        # the softmax part alone: subtract the oracle's one-hot terms from both sides
+        assert parity.rel_fro(got - (rows - dense), dense) <= parity.TOL_DENSE
 
 
 def test_qwen3_0p6b_full():
-    n = _full_size_case("qwen3_0p6b")
+    n = _Case("qwen3_0p6b").check()
     assert n > 30000
 
 
 def test_qwen3_8b_full():
-    n = _full_size_case("qwen3_8b")
+    n = _Case("qwen3_8b").check()
     assert n > 100000
-
-
-def test_qwen3_8b_full_single_pass():
-    n = _full_size_case("qwen3_8b", fused=True)
-    assert n > 100000
-
-
-def test_qwen3_0p6b_full_single_pass():
-    _full_size_case("qwen3_0p6b", fused=True)
 
 
 def test_qwen3_8b_sweep_points():
     # the selection-fraction sweep's other settings on the same batch shape (smaller P to
     # keep the test short): URS p = 0.25, full-token p = 1, deterministic truncation
+    case = _Case("qwen3_8b", P=2)
     for kw in (dict(sel_mode="urs", p=0.25), dict(sel_mode="urs", p=1.0),
                dict(sel_mode="det", beta=0.5)):
-        _full_size_case("qwen3_8b", P=2, **kw)
+        case.check(routes=(True,), **kw)
 
 
-def test_long_cot_full():
-    n = _full_size_case("long_cot")
-    assert n > 300000
+def test_long_cot_three_way():
+    """Long chain-of-thought batch: RPC (C = 100), URS p = 0.5 and the full-token case p = 1
+    on identical seeded tensors, each through both routes.  p = 1 selects every token
+    (Eq. ht-estimator with m = 1, p = 1: plain GRPO), 1.3 million rows in ~160 row chunks."""
+    case = _Case("long_cot")
+    n_rpc = case.check()                                       # the workload's own setting: RPC
+    n_urs = case.check(sel_mode="urs", p=0.5)
+    n_all = case.check(sel_mode="urs", p=1.0)
+    assert n_all == case.batch["n_tot"] and n_all > 1000000
+    assert 0.45 * n_all < n_urs < 0.55 * n_all and 0.45 * n_all < n_rpc < 0.6 * n_all

@@ -50,11 +50,27 @@ def test_mid_bf16_multi_chunk_shapes():
 
 
 def test_twin_0p6b():
-    parity.run_case(wl.WORKLOADS["twin_0p6b"], seed=0)
+    parity.run_case(wl.WORKLOADS["twin_0p6b"], seed=0, routes=(False, True))
 
 
 def test_twin_8b():
-    parity.run_case(wl.WORKLOADS["twin_8b"], seed=0)
+    parity.run_case(wl.WORKLOADS["twin_8b"], seed=0, routes=(False, True))
+
+
+@pytest.mark.parametrize("name,w_scale", [("twin_0p6b", 0.5), ("twin_8b", 0.15), ("twin_8b", 0.5)])
+def test_twins_with_peaked_softmax(name, w_scale):
+    """The real heads (d = 1024 / 4096, V = 151936) with logits of standard deviation 16,
+    ~10 and 32 instead of ~1: the softmax part of the gradients is then as large as the
+    one-hot part, so the dense-part comparison of dHidden is not hidden behind bf16
+    rounding, and the running-max rescaling of the forward is exercised.  (At standard
+    deviation 32 a row's largest logit can exceed the single-pass window above its
+    reference; the single-pass call then redoes the chunk with the two-pass kernels.)"""
+    w = wl.variant(wl.WORKLOADS[name], w_scale=w_scale, old_noise=0.3)
+    out, ref = parity.run_case(w, seed=1, routes=(False, True))
+    resolv = 2.0 ** -9 * np.linalg.norm(ref["dH"]) / np.linalg.norm(ref["dH_dense"])
+    assert resolv < 5e-3                       # the bf16 slack is small here: the check bites
+    assert out["dH_dense_err"] <= parity.TOL_DENSE
+    assert out["status"] & ~nat.NAT_DEV_FALLBACK == 0
 
 
 def test_accumulate_dW_and_dloss():
@@ -88,10 +104,11 @@ def test_empty_selection_and_reruns_are_deterministic():
     w = wl.WORKLOADS["mid"]
     batch = wl.make_batch(w, seed=0, device="cuda")
     st = parity.gpu_step(w, batch, 0, 0)
-    loss1, logp1 = st.loss.clone(), st.logp.clone()
+    loss1, logp1, dW1 = st.loss.clone(), st.logp.clone(), st.dW.clone()
     st.run(batch, w.sel_mode, p=w.p, seed=0)
     torch.cuda.synchronize()
     assert torch.equal(loss1, st.loss) and torch.equal(logp1, st.logp)
+    assert torch.equal(dW1, st.dW)
     # nothing selected: loss 0 and zero dW
     st.mask.zero_()
     st.compact(batch["cu_seqlens"])
@@ -123,7 +140,7 @@ def test_unsupported_shapes_are_rejected():
 
 
 # ---- single-pass route: nat_policy_loss_fwd_bwd ------------------------------------
-@pytest.mark.parametrize("name", ["tiny", "mid", "twin_0p6b", "twin_8b"])
+@pytest.mark.parametrize("name", ["tiny", "mid"])
 def test_fused_matches_oracle(name):
     parity.run_case(wl.WORKLOADS[name], seed=0, fused=True)
 
@@ -202,12 +219,13 @@ def test_fused_empty_selection_capacity_and_reruns():
     batch = wl.make_batch(w, seed=0, device="cuda")
     args = (batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], batch["cu_seqlens"])
     st = parity.gpu_step(w, batch, 0, 0, fused=True)
-    loss1, logp1, dH1 = st.loss.clone(), st.logp.clone(), st.dH.clone()
+    loss1, logp1, dH1, dW1 = st.loss.clone(), st.logp.clone(), st.dH.clone(), st.dW.clone()
     st.run(batch, w.sel_mode, p=w.p, seed=0, fused=True)
     torch.cuda.synchronize()
     n = int(st.n_sel.item())
     assert torch.equal(loss1, st.loss) and torch.equal(logp1[:n], st.logp[:n])
-    assert torch.equal(dH1[:n], st.dH[:n])            # dense parts are order-fixed
+    assert torch.equal(dH1[:n], st.dH[:n])            # every sum has a fixed order
+    assert torch.equal(dW1, st.dW)
     # nothing selected: loss 0 and zero dW
     st.mask.zero_()
     st.compact(batch["cu_seqlens"])
@@ -261,3 +279,53 @@ def test_kl_term(name, fused):
     # kl_beta != 0 without a reference is refused
     with pytest.raises(nat.NatError):
         parity.gpu_step(w, batch, 5, 0, fused=fused, kl_beta=0.05, ref_logp=None)
+
+
+def test_dW_is_reproducible_when_many_tokens_share_a_target():
+    # 40 distinct targets over ~800 selected tokens: every target row of dW receives some
+    # twenty one-hot terms, whose order of summation must not depend on the run
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=7, device="cuda")
+    batch["targets"] = (batch["targets"] % 40).to(torch.int32)
+    batch["old_logp"] = wl.library_logp(batch["hidden"], batch["W"], batch["targets"]) + \
+        0.05 * torch.randn(batch["n_tot"], device="cuda")
+    nb = wl.to_numpy(batch)
+    ref_sel = parity.oracle_selection(w, nb, 7, 0)
+    ref = None
+    for fused in (False, True):
+        st = parity.gpu_step(w, batch, 7, 0, fused=fused)
+        out, ref = parity.check_loss(st, ref_sel, nb, w, ref=ref)
+        dW1 = st.dW.clone()
+        for _ in range(3):
+            st.run(batch, w.sel_mode, p=w.p, seed=7, fused=fused)
+            torch.cuda.synchronize()
+            assert torch.equal(dW1, st.dW)
+
+
+def test_target_outside_the_vocabulary_is_reported_and_left_out():
+    w = wl.WORKLOADS["mid"]
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    nb = wl.to_numpy(batch)
+    ref_sel = parity.oracle_selection(w, nb, 0, 0)
+    bad = ref_sel["sel_idx"][[3, 200]]
+    clean = {}
+    for fused in (False, True):
+        st = parity.gpu_step(w, batch, 0, 0, fused=fused)
+        clean[fused] = (st.dW.clone(), st.dH.clone(), st.logp.clone())
+    targets = batch["targets"].clone()
+    targets[int(bad[0])] = w.V + 5
+    targets[int(bad[1])] = -1
+    poisoned = dict(batch, targets=targets)
+    for fused in (False, True):
+        st = parity.gpu_step(w, poisoned, 0, 0, fused=fused)
+        assert st.status() & nat.NAT_DEV_BAD_TARGET
+        n = ref_sel["n_sel"]
+        logp = st.logp[:n]
+        assert torch.isnan(logp[3]) and torch.isnan(logp[200]) and int(torch.isnan(logp).sum()) == 2
+        assert torch.all(st.dH[3] == 0) and torch.all(st.dH[200] == 0)
+        keep = torch.ones(n, dtype=torch.bool, device="cuda")
+        keep[3] = keep[200] = False
+        assert torch.equal(st.dH[:n][keep], clean[fused][1][:n][keep])
+        assert torch.isfinite(st.dW).all() and torch.isfinite(st.loss).all()
+    # a clean batch leaves the bit clear
+    assert parity.gpu_step(w, batch, 0, 0, fused=True).status() & nat.NAT_DEV_BAD_TARGET == 0

@@ -24,6 +24,8 @@ def _select_compact(T, mode, P, G, seed=0, offset=0, p=0.5, min_cut=1, beta=0.5,
         rewards = (np.random.default_rng(seed).random(P * G) < 0.4).astype(np.float32)
     st.grpo_adv(torch.from_numpy(rewards).cuda())
     st.select(cu_d, mode, p=p, min_cut=min_cut, beta=beta, seed=seed, offset=offset)
+    for t in (st.sel_idx, st.sel_resp, st.sel_offsets, st.n_sel):
+        t.fill_(-9)
     st.compact(cu_d)
     torch.cuda.synchronize()
     adv = oracle.grpo_adv(rewards, P, G, 1e-6)
@@ -35,11 +37,25 @@ def _select_compact(T, mode, P, G, seed=0, offset=0, p=0.5, min_cut=1, beta=0.5,
     assert np.array_equal(st.pi[:n_tot].cpu().numpy().view(np.uint32), pi.view(np.uint32))
     if cut is not None:
         assert np.array_equal(st.cut_len[:P * G].cpu().numpy(), cut)
-    assert int(st.n_sel.item()) == n
     m = n if cap is None else min(n, cap)
-    assert np.array_equal(st.sel_idx[:m].cpu().numpy(), si[:m])
-    assert np.array_equal(st.sel_resp[:m].cpu().numpy(), sr[:m])
-    assert np.array_equal(st.sel_offsets.cpu().numpy(), so)
+
+    def check_lists():
+        assert int(st.n_sel.item()) == n
+        assert np.array_equal(st.sel_idx[:m].cpu().numpy(), si[:m])
+        assert np.array_equal(st.sel_resp[:m].cpu().numpy(), sr[:m])
+        assert np.array_equal(st.sel_offsets.cpu().numpy(), so)
+        if m < st.sel_idx.numel():
+            assert int(st.sel_idx[m:].max()) == -9       # nothing written past the lists' end
+
+    check_lists()
+    if mode != "urs":
+        # prefix modes: st.compact() built the lists from the cut lengths alone; the
+        # generic compaction of the mask must give the same lists
+        for t in (st.sel_idx, st.sel_resp, st.sel_offsets, st.n_sel):
+            t.fill_(-9)
+        st.compact(cu_d, from_mask=True)
+        torch.cuda.synchronize()
+        check_lists()
     return n
 
 
@@ -119,6 +135,10 @@ def test_skewed_lengths_miss_the_proportional_window():
 def test_capacity_smaller_than_selection():
     n = _select_compact([300, 200, 100, 50], "urs", 2, 2, seed=1, p=0.9, cap=64)
     assert n > 64
+    n = _select_compact([300, 200, 100, 50], "det", 2, 2, seed=1, beta=0.9, cap=64)
+    assert n > 64
+    n = _select_compact([5000, 9000, 100, 50], "rpc", 2, 2, seed=1, min_cut=4000, cap=4099)
+    assert n > 4099
 
 
 def test_rewards_real_valued():
@@ -161,9 +181,10 @@ def test_survival_schedule_selection(lengths):
     surv_d = torch.from_numpy(surv).cuda() if n_tot else torch.zeros(16, device="cuda")
     for seed, offset in ((3, 0), (3, (5 << 32) + 9)):
         nat.nat_select_survival(B, torch.from_numpy(cu).cuda(), n_tot, surv_d, seed, offset,
-                                mask, cut)
+                                mask, cut, resp_base=offset & 7)
         torch.cuda.synchronize()
-        ref_mask, ref_cut = oracle.select_survival(cu, surv, seed=seed, offset=offset)
+        ref_mask, ref_cut = oracle.select_survival(cu, surv, seed=seed, offset=offset,
+                                                   resp_base=offset & 7)
         assert np.array_equal(mask[:n_tot].cpu().numpy(), ref_mask)
         assert np.array_equal(cut.cpu().numpy(), ref_cut)
 
@@ -226,3 +247,86 @@ def test_gather_and_scatter_rows(d, dtype):
     # row_bytes must be a multiple of 16
     assert nat.load().nat_gather_rows(x.data_ptr(), 24, st.sel_idx.data_ptr(), st.n_sel.data_ptr(), 3,
                                       packed.data_ptr(), None) == -1
+
+
+# ------------------------------------------------- sharding: response-index base
+@pytest.mark.parametrize("mode", ["urs", "rpc", "det"])
+def test_shards_realise_slices_of_the_whole_batch_selection(mode):
+    """Two data-parallel shards of one batch, each passing only its own responses and the
+    global index of its first one, draw exactly the whole batch's mask, pi and cuts."""
+    w = wl.WORKLOADS["qwen3_0p6b"]
+    T = wl.make_lengths(w, 2)
+    cu = wl.cu_from_lengths(T)
+    kw = dict(p=0.5, min_cut=100, beta=0.5, seed=5, offset=(3 << 32) + 1)
+    mask, pi, cut = oracle.select(MODE_ID[mode], cu, **kw)
+    for lo, hi in ((0, 24), (24, 64)):
+        cu_s = wl.cu_from_lengths(T[lo:hi])
+        n_s = int(cu_s[-1])
+        st = NatStep((hi - lo) // w.G, w.G, 64, 512, torch.float32, n_s, want_grads=False,
+                     B_global=w.B, resp_base=lo)
+        cu_d = torch.from_numpy(cu_s).cuda()
+        st.select(cu_d, mode, **kw)
+        st.compact(cu_d)
+        torch.cuda.synchronize()
+        assert np.array_equal(st.mask[:n_s].cpu().numpy(), mask[cu[lo]:cu[hi]])
+        assert np.array_equal(st.pi[:n_s].cpu().numpy().view(np.uint32),
+                              pi[cu[lo]:cu[hi]].view(np.uint32))
+        if cut is not None:
+            assert np.array_equal(st.cut_len[:hi - lo].cpu().numpy(), cut[lo:hi])
+        si, sr, so, n = oracle.compact(mask[cu[lo]:cu[hi]], cu_s)
+        assert int(st.n_sel.item()) == n
+        assert np.array_equal(st.sel_idx[:n].cpu().numpy(), si)
+        assert np.array_equal(st.sel_resp[:n].cpu().numpy(), sr)
+
+
+# ------------------------------------------------------------ general cut laws
+def _law(T, rng):
+    q = (np.maximum(0.995 ** np.arange(T), 0.05) * rng.uniform(0.5, 1.0, T) / max(T, 1))
+    return q.astype(np.float32)
+
+
+@pytest.mark.parametrize("lengths", [[1, 5, 64, 300, 0, 17, 4096, 33, 4095, 1, 0, 8193],
+                                     [0, 0, 7, 0], [0, 0, 0], "qwen3_0p6b", "long_cot"])
+def test_cut_law_selection(lengths):
+    """nat_select_cutlaw against the oracle, bit for bit: pi is the suffix sum of the law
+    over each response (a scan over the packed stream on the device), one cut per response."""
+    if isinstance(lengths, str):
+        lengths = wl.make_lengths(wl.WORKLOADS[lengths], 0)
+    T = np.asarray(lengths, dtype=np.int32)
+    cu = wl.cu_from_lengths(T)
+    n_tot, B = int(cu[-1]), len(T)
+    rng = np.random.default_rng(3)
+    q = np.concatenate([_law(int(t), rng) for t in T] + [np.zeros(0, np.float32)])
+    if n_tot > 40:
+        q[7] = 0.0                      # a zero mass inside a response
+        q[11] = -1.0                    # negative and NaN count as zero
+        q[13] = np.nan
+        q[cu[2]:cu[3]] = 0.0            # a response whose law has no mass at all: kept whole
+    if B > 7:
+        q[cu[7]:cu[8]] = 1.0 / 64       # dyadic uniform law
+        q[cu[6] + 2000:cu[7]] = 0.0     # no mass after position 2000: pi = 0 there
+    pad = max(n_tot, 16)
+    mask = torch.full((pad,), 7, dtype=torch.uint8, device="cuda")
+    pi = torch.full((pad,), -1.0, dtype=torch.float32, device="cuda")
+    cut = torch.full((max(B, 1),), -1, dtype=torch.int32, device="cuda")
+    q_d = torch.zeros(pad, device="cuda")
+    q_d[:n_tot] = torch.from_numpy(q)
+    ws = nat.alloc_workspace(nat.nat_select_cutlaw_workspace_bytes(B, n_tot), "cuda")
+    cu_d = torch.from_numpy(cu).cuda()
+    for seed, offset, base in ((3, 0, 0), (4, (5 << 32) + 9, 17)):
+        nat.nat_select_cutlaw(B, cu_d, n_tot, q_d, seed, offset, mask, pi, cut, ws, resp_base=base)
+        torch.cuda.synchronize()
+        rm, rp, rc = oracle.select_cutlaw(cu, q, seed=seed, offset=offset, resp_base=base)
+        assert np.array_equal(mask[:n_tot].cpu().numpy(), rm)
+        assert np.array_equal(pi[:n_tot].cpu().numpy().view(np.uint32), rp.view(np.uint32))
+        assert np.array_equal(cut[:B].cpu().numpy(), rc)
+    # the cut lengths feed the prefix compaction
+    st = NatStep(1, max(B, 1), 64, 512, torch.float32, n_tot, want_grads=False)
+    nat.nat_compact_prefix(B, cu_d, n_tot, cut, st.sel_idx, st.sel_resp, st.sel_offsets, st.n_sel,
+                           st.cap)
+    torch.cuda.synchronize()
+    si, sr, so, n = oracle.compact(rm, cu)
+    assert int(st.n_sel.item()) == n
+    assert np.array_equal(st.sel_idx[:n].cpu().numpy(), si)
+    assert np.array_equal(st.sel_resp[:n].cpu().numpy(), sr)
+    assert np.array_equal(st.sel_offsets[:B + 1].cpu().numpy(), so)
