@@ -4,15 +4,30 @@
 
 A step is one pass of the whole path over one synthetic batch: advantages,
 selection, compaction, policy-loss forward and backward (by default through the
-single-pass call nat_policy_loss_fwd_bwd; --route two times the separate calls).  Rank 0 prints ONE
-JSON line.  `value` is selected tokens per second with inputs resident in HBM;
+single-pass call nat_policy_loss_fwd_bwd; --route two times the separate calls).  Rank 0
+prints ONE JSON line.  `value` is selected tokens per second with inputs resident in HBM;
 `e2e` is the same with the step's inputs copied from pinned host memory and the
 loss read back inside the timed region.  `--impl reference` times the fp64 CPU
 oracle on a bounded sample of the same workload.
+
+With --gpus N > 1 and no torchrun environment the script starts the N ranks itself (one
+process per GPU).  By default the ranks run independent batches (weak scaling, no
+collective on the data path); --sharded makes them split ONE batch by prompt groups and
+sum loss and dW with an all-reduce every step (the exchange of a data-parallel trainer).
+
+Other measurements (markdown tables on stdout instead of the JSON line):
+    --mode sweep     time against the selected-token fraction (URS p, RPC, truncation)
+    --mode stress    selection / compaction / packing GB/s on a 2^28-token stream
+    --mode ceiling   the loss kernels against the library's plain GEMMs on the same operands
+    --mode source-hash   hash of the tensor-core kernel sources (ties ncu counters to a build)
 """
 import argparse
+import glob
+import hashlib
 import json
 import os
+import re
+import socket
 import statistics
 import subprocess
 import sys
@@ -26,6 +41,8 @@ if ROOT not in sys.path:
 METRIC = "selected tokens/sec, fused policy-loss fwd+bwd (Qwen3-8B head); % bf16 TC peak"
 UNIT = "selected tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "nat_tc_kernel_dram_traffic.json")
+KERNEL_SOURCES = ("nat_loss_bf16.cu", "nat_tc.cuh")
 
 
 def load_peaks():
@@ -35,6 +52,31 @@ def load_peaks():
             p = json.load(f)
         return p, "measured"
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def kernel_source_hash():
+    """sha256 over the sources of the tensor-core loss kernels: the ncu counters kept under
+    profiles/ carry the hash of the sources they were taken from."""
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2603_06619_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def dram_traffic(kind, d, V, chunk_rows):
+    """DRAM bytes per launch of one loss kernel from the tracked ncu capture, or (None, why)
+    when no capture covers this shape or the kernels changed after it was taken."""
+    if not os.path.exists(TRAFFIC_FILE):
+        return None, "no capture on file"
+    with open(TRAFFIC_FILE) as f:
+        t = json.load(f)
+    if t.get("source_hash") != kernel_source_hash():
+        return None, "kernel sources changed since the counters were taken"
+    for c in t.get("captures", []):
+        if (c["kernel"], c["d"], c["V"], c["chunk_rows"]) == (kind, d, V, chunk_rows):
+            return c["dram_bytes_per_launch"], c.get("summary", "")
+    return None, "shape not covered by the capture"
 
 
 class ClockSampler:
@@ -72,7 +114,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             if len(r) < 7:
@@ -80,13 +122,15 @@ class ClockSampler:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
+                pw.append(float(r[2]))
             except ValueError:
                 continue
             for name, val in zip(names, r[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None,
-                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w": statistics.median(pw) if pw else None, "reasons": sorted(reasons),
                 "samples": len(sm)}
 
 
@@ -95,6 +139,30 @@ def host_cores():
         return len(os.sched_getaffinity(0))
     except AttributeError:
         return os.cpu_count()
+
+
+def pick_workload(args):
+    """The named workload with the command line's overrides (selection, prompt count)."""
+    from paper_2603_06619_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    if args.prompts:
+        w = wl.variant(w, P=args.prompts)
+    if args.selection:
+        mode, _, val = args.selection.partition(":")
+        if mode == "urs":
+            w = wl.variant(w, sel_mode="urs", p=float(val or 0.5))
+        elif mode == "rpc":
+            w = wl.variant(w, sel_mode="rpc", min_cut=int(val or 100))
+        elif mode == "det":
+            w = wl.variant(w, sel_mode="det", beta=float(val or 0.5))
+        else:
+            raise SystemExit("--selection takes urs:P, rpc:C or det:BETA")
+    return w
+
+
+def selection_label(w):
+    return {"urs": f"URS p={w.p:g}", "rpc": f"RPC C={w.min_cut}",
+            "det": f"deterministic truncation beta={w.beta:g}"}[w.sel_mode]
 
 
 # ---------------------------------------------------------------- CPU oracle
@@ -126,8 +194,6 @@ def run_reference(args, w):
     if rank != 0:
         return
     rows = args.ref_rows
-    for _ in range(args.warmup):
-        pass  # the oracle has no warm state worth building; keep the run short
     rate, _, n, times = oracle_sample_rate(w, seed=0, rows=rows, repeats=max(1, args.steps))
     ms = 1e3 * statistics.mean(times)
     cores = host_cores()
@@ -146,12 +212,59 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------ launcher
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launcher_command(n, argv, port):
+    """The command that starts `n` ranks of this script on one node (one process per GPU)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node",
+            str(n), "--master-addr", "127.0.0.1", "--master-port", str(port),
+            os.path.abspath(__file__)] + list(argv)
+
+
+def launch_ranks(args, argv):
+    """--gpus N given to a plain `python bench.py`: start the N ranks and pass rank 0's JSON
+    line through.  NCCL's communicator log goes to a file per rank so that stdout stays one
+    line; rank 0 reads the rank count back from it into the line."""
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("NCCL_DEBUG_FILE", f"/tmp/nat_bench_nccl_{os.getpid()}.%h.%p.log")
+    cmd = launcher_command(args.gpus, argv, free_port())
+    return subprocess.call(cmd, env=env)
+
+
+def nccl_log_summary():
+    """Rank count and NVLS use as NCCL's own log states them (None when no log was kept)."""
+    pattern = os.environ.get("NCCL_DEBUG_FILE")
+    if not pattern:
+        return None
+    path = pattern.replace("%h", socket.gethostname()).replace("%p", str(os.getpid()))
+    files = [path] if os.path.exists(path) else glob.glob(re.sub(r"%[hp]", "*", pattern))
+    nranks, nvls = None, False
+    for fpath in files[:8]:
+        try:
+            text = open(fpath, errors="replace").read()
+        except OSError:
+            continue
+        m = re.findall(r"nranks (\d+)", text)
+        if m:
+            nranks = max(int(x) for x in m)
+        nvls = nvls or ("NVLS" in text and "NVLS multicast support is available" in text)
+    return {"nranks": nranks, "nvls": nvls, "log": pattern}
+
+
 # --------------------------------------------------------------------- ours
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
 
     from paper_2603_06619_b200 import build as _build
+    from paper_2603_06619_b200 import nat as _nat
     from paper_2603_06619_b200 import sharding
     from paper_2603_06619_b200 import workloads as wl
     from paper_2603_06619_b200.step import NatStep
@@ -159,6 +272,9 @@ def run_ours(args, w):
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if local_rank >= torch.cuda.device_count():
+        raise SystemExit(f"rank {rank}: no GPU {local_rank} (this node shows "
+                         f"{torch.cuda.device_count()}); --gpus must not exceed the GPUs present")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if world > 1:
@@ -168,18 +284,36 @@ def run_ours(args, w):
     if world > 1:
         dist.barrier()
 
-    # Responses are independent, so ranks take disjoint batches (weak scaling):
-    # no collective sits on the data path.
-    seed = sharding.rank_seed(args.seed, rank)
-    batch = wl.make_batch(w, seed=seed, device=dev)
+    sharded = args.sharded and world > 1
+    exchange_on = sharded or (args.allreduce_dw and world > 1)
+    if sharded:
+        # ONE batch, split by prompt groups: this rank holds responses [lo, hi) of it, keeps
+        # the batch's size as the divisor of the batch mean and draws its masks with the
+        # global response indices; W is the same on every rank.
+        seed = args.seed
+        T_all = wl.make_lengths(w, seed)
+        lo, hi = sharding.response_range(w.P, w.G, rank, world)
+        if hi == lo:
+            raise SystemExit(f"--sharded needs at least one prompt per rank (P = {w.P}, {world} ranks)")
+        w_local = wl.variant(w, P=(hi - lo) // w.G)
+        batch = wl.make_batch(w_local, seed=seed + 1000 * (rank + 1), device=dev,
+                              lengths=T_all[lo:hi], W_seed=seed)
+        step_kw = dict(B_global=w.B, resp_base=lo)
+    else:
+        # Responses are independent, so ranks take disjoint batches (weak scaling):
+        # no collective sits on the data path.
+        seed = sharding.rank_seed(args.seed, rank)
+        w_local = w
+        batch = wl.make_batch(w, seed=seed, device=dev)
+        step_kw = {}
     n_tot = batch["n_tot"]
     dtype = torch.float32 if w.dtype == "f32" else torch.bfloat16
-    st = NatStep(w.P, w.G, w.d, w.V, dtype, n_tot, device=dev)
+    st = NatStep(w_local.P, w_local.G, w.d, w.V, dtype, n_tot, device=dev, **step_kw)
     cu = batch["cu_seqlens"]
-    sel = dict(mode=w.sel_mode, p=w.p, min_cut=w.min_cut, beta=w.beta, seed=seed)
+    sel = dict(mode=w.sel_mode, p=w.p, min_cut=w.min_cut, beta=w.beta, seed=args.seed if sharded else seed)
 
     def exchange():
-        if args.allreduce_dw and world > 1:
+        if exchange_on:
             sharding.allreduce_grads(st.loss, st.dW)
 
     def step(b, offset):
@@ -240,8 +374,16 @@ def run_ours(args, w):
     elapsed_ms = t_begin.elapsed_time(t_end)
     loss_call_ms = statistics.mean(e[0].elapsed_time(e[2]) for e in ev)
     first_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    prep_ms = (elapsed_ms - sum(e[0].elapsed_time(e[2]) for e in ev)) / args.steps
     status = st.status()
     loss_val = float(st.loss.item())
+    if args.only_steps:
+        if rank == 0:
+            print(json.dumps({"only_steps": True, "workload": w.name, "steps": args.steps,
+                              "ms_per_step": elapsed_ms / args.steps, "device_status": status}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     # selected tokens per step: selection with offsets warmup..warmup+K-1 (replayed, untimed)
     n_sel_total = 0
     for i in range(args.steps):
@@ -251,7 +393,6 @@ def run_ours(args, w):
 
     # ---- per-kernel durations: the same K steps again with event pairs around every
     # tensor-core launch (kept out of the timed region above)
-    from paper_2603_06619_b200 import nat as _nat
     trace = None
     if w.dtype == "bf16":
         _nat.nat_trace_begin()
@@ -337,19 +478,21 @@ def run_ours(args, w):
     executed = counted if args.route == "single" else 8.0 * n_step * dV
     call_tflops = counted / (loss_call_ms * 1e-3) / 1e12
     step_tflops = counted / (step_ms * 1e-3) / 1e12
-    cap_pad = (n_tot + 255) // 256 * 256
-    n_chunks = (cap_pad + min(cap_pad, 8192) - 1) // min(cap_pad, 8192)
-    sel_launches = 1 + (1 if w.sel_mode == "urs" else 2) + 3
+    cap_pad = (n_tot + 511) // 512 * 512
+    chunk_rows = min(cap_pad, 8192)
+    n_chunks = (cap_pad + chunk_rows - 1) // chunk_rows
+    sel_launches = 1 + (1 if w.sel_mode == "urs" else 2) + (3 if w.sel_mode == "urs" else 2)
     if w.dtype == "f32":
         launches = sel_launches + 2 + 3
     elif args.route == "single":
-        launches = sel_launches + 2 + 9 * n_chunks + 3      # gather, references; per chunk 9; tail 3
+        # gather, references; per chunk 9; tail: fallback note, 5 one-hot kernels, loss sum
+        launches = sel_launches + 2 + 9 * n_chunks + 7
     else:
-        launches = sel_launches + 4 + (3 + 3 * n_chunks)
+        launches = sel_launches + 3 + (2 + 3 * n_chunks + 5)
     kernel = ("nat_tc_kernel<kE|kDh|kDw> (the launches inside nat_policy_loss_fwd_bwd)"
               if args.route == "single" else
               "nat_tc_kernel<kFwd|kDz|kDh|kDw> (nat_policy_loss_fwd + nat_policy_loss_bwd)")
-    roof_ms, roof_flops, per_kernel, traffic = loss_call_ms, counted, None, None
+    roof_ms, roof_flops, per_kernel, traffic, traffic_note = loss_call_ms, counted, None, None, None
     if trace:
         # counted FLOPs of one step per kernel kind: the forward's 2NdV belongs to kFwd or kE,
         # dH and dW have 2NdV each, the recompute (kDz) and the one-tile reference pass have none
@@ -371,33 +514,42 @@ def run_ours(args, w):
         kernel = "nat_tc_kernel<%s>" % {"e": "kE", "dh": "kDh", "dw": "kDw", "dz": "kDz",
                                          "fwd": "kFwd"}[top]
         roof_ms, roof_flops = per_kernel[top]["ms_per_step"], credit[top]
-        # DRAM bytes per launch (one 8192-row chunk of this head) from the ncu capture
-        # summarised in profiles/nat_tc_kernel_qwen3_8b_chunk.md; null for other shapes
-        if w.name == "qwen3_8b":
-            traffic = {"e": 9.51e9, "dh": 16.79e9, "dw": 21.37e9}.get(top)
+        # DRAM bytes per launch (one row chunk of this head) from the tracked ncu capture
+        traffic, traffic_note = dram_traffic(top, w.d, w.V, chunk_rows)
     call_tflops = roof_flops / (roof_ms * 1e-3) / 1e12
+    sm_mhz = clocks.get("sm_mhz") if clocks else None
 
+    if sharded:
+        parallelism = (f"dp{world}: one batch of {w.B} responses split by prompt groups, loss and "
+                       "dW all-reduced (NCCL) every step")
+    elif exchange_on:
+        parallelism = f"dp{world} (independent batches, loss and dW all-reduced every step)"
+    else:
+        parallelism = f"dp{world} (independent batches, no collective)"
     line = {
         "metric": METRIC, "value": n_all / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": w.name, "P": w.P, "G": w.G, "d": w.d, "V": w.V,
-                   "selection": w.sel_mode, "p": w.p, "min_cut": w.min_cut,
+                   "selection": w.sel_mode, "p": w.p, "min_cut": w.min_cut, "beta": w.beta,
+                   "selection_label": selection_label(w),
                    "route": ("single pass (nat_policy_loss_fwd_bwd)" if args.route == "single"
                              else "two pass (nat_policy_loss_fwd, nat_policy_loss_bwd)"),
                    "n_tot_per_gpu": n_tot, "n_sel_per_step_per_gpu": n_step,
-                   "l2": "inputs larger than L2 (hidden and W_lm are GBs); no flush needed",
-                   "parallelism": (f"dp{world} (independent batches, loss and dW all-reduced "
-                                   "every step)" if args.allreduce_dw and world > 1 else
-                                   f"dp{world} (independent batches, no collective)")},
+                   "l2": "inputs larger than L2 (hidden and W_lm are GBs); no flush needed"
+                   if n_tot * w.d * 2 > 2 * 126e6 else
+                   "W_lm (hundreds of MB) and the numerator scratch exceed L2; hidden does not",
+                   "parallelism": parallelism},
         "tflops_counted": step_tflops,
         "tflops_executed": executed / (step_ms * 1e-3) / 1e12,
         "frac_of_peak_counted": {
             "burst": step_tflops / float(peaks["bf16_tflops"]),
             "sustained": step_tflops / peak,
             "datasheet_2250": step_tflops / 2250.0},
-        "loss_call_ms": loss_call_ms, "loss": loss_val, "device_status": status,
+        "loss_call_ms": loss_call_ms, "select_compact_adv_ms": prep_ms, "loss": loss_val,
+        "device_status": status,
+        "ms_times_sm_mhz": step_ms * sm_mhz if sm_mhz else None,
         "other_route": None if args.skip_other_route else {
             "route": "two pass" if args.route == "single" else "single pass",
             "ms_per_step": other_ms / args.steps,
@@ -410,15 +562,21 @@ def run_ours(args, w):
             "flops": ("counted 2*N_sel*d*V per step for this kernel, divided by its event-timed "
                       "duration summed over the step's launches (nat_trace_begin/end)") if trace
             else "counted 6*N_sel*d*V per step divided by the event-timed loss call(s)",
-            "traffic": traffic, "traffic_unit": "DRAM bytes per launch (8192-row chunk)"},
+            "traffic": traffic, "traffic_unit": "DRAM bytes per launch (one row chunk)",
+            "traffic_source": traffic_note},
         "per_kernel": per_kernel,
         "e2e": {"value": n_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": 4, "ms_per_step": e2e_ms / args.steps,
                 "pipeline": "step i+1's inputs are copied on a second stream (two device buffer "
-                            "sets) while step i computes; all copies inside the timed region"},
+                            "sets) while step i computes; all copies inside the timed region",
+                "stays_on_device": "W_lm is resident; of the results only the loss scalar returns "
+                                   "to the host: dHidden and dW stay in HBM, where a trainer's "
+                                   "backward pass and optimizer consume them"},
         "gpu_launches": launches * args.steps,
         "clocks": clocks,
     }
+    if world > 1:
+        line["nccl"] = nccl_log_summary()
     if args.route == "two":
         line["fwd_ms"], line["bwd_ms"] = first_ms, loss_call_ms - first_ms
     if not args.no_cpu_baseline and world == 1:
@@ -432,30 +590,299 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------- other measurements
+def _time(fn, reps, warmup=1):
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def fraction_sweep(w, reps=2, seed=0):
+    """The single-pass loss on one batch under every selection setting of the sweep (URS
+    p = 0.25 .. 1, RPC with the paper's minimum cut of 100, deterministic 50 % truncation)
+    and the fit time = a + b * fraction."""
+    import numpy as np
+    import torch
+    from paper_2603_06619_b200 import workloads as wl
+    from paper_2603_06619_b200.step import NatStep
+
+    batch = wl.make_batch(w, seed=seed, device="cuda")
+    n_tot = batch["n_tot"]
+    st = NatStep(w.P, w.G, w.d, w.V, torch.bfloat16, n_tot)
+    cu = batch["cu_seqlens"]
+    st.grpo_adv(batch["rewards"])
+    settings = [("URS p=0.25", dict(mode="urs", p=0.25)), ("URS p=0.5", dict(mode="urs", p=0.5)),
+                ("URS p=0.75", dict(mode="urs", p=0.75)),
+                ("full tokens (URS p=1)", dict(mode="urs", p=1.0)),
+                ("RPC C=100", dict(mode="rpc", min_cut=100)),
+                ("Det. trunc. 50%", dict(mode="det", beta=0.5))]
+    peaks, kind = load_peaks()
+    rows = []
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    for label, kw in settings:
+        st.select(cu, seed=seed, **kw)
+        st.compact(cu)
+        n_sel = int(st.n_sel.item())
+        args = (batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+        ms = _time(lambda: st.loss_fwd_bwd(*args), reps)
+        assert st.status() & ~4 == 0
+        tf = 6.0 * n_sel * w.d * w.V / (ms * 1e-3) / 1e12
+        rows.append((label, n_sel, n_sel / n_tot, ms, tf))
+    clocks = sampler.stop()
+    x = np.array([r[2] for r in rows])
+    y = np.array([r[3] for r in rows])
+    b, a = np.polyfit(x, y, 1)
+    resid = y - (a + b * x)
+    out = [f"Workload {w.name}: N_tot = {n_tot}, d = {w.d}, V = {w.V}; single-pass "
+           f"nat_policy_loss_fwd_bwd, mean of {reps} calls after 1 warm-up; peaks {kind}; SM clock "
+           f"median {clocks['sm_mhz']} MHz, reasons {clocks['reasons']}.", "",
+           "| selection | n_sel | fraction | ms | TFLOP/s counted | of burst peak | of sustained peak |",
+           "|---|---|---|---|---|---|---|"]
+    for label, n_sel, frac, ms, tf in rows:
+        out.append(f"| {label} | {n_sel} | {frac:.3f} | {ms:.1f} | {tf:.0f} | "
+                   f"{tf / peaks['bf16_tflops']:.3f} | {tf / peaks['bf16_tflops_sustained']:.3f} |")
+    out += ["", f"Least-squares fit: time = a + b * fraction with a = {a:.1f} ms, b = {b:.1f} ms "
+            f"(a/b = {a / b:.3f}); largest residual {np.abs(resid).max():.1f} ms "
+            f"({100 * np.abs(resid / y).max():.1f} % of its point)."]
+    return "\n".join(out)
+
+
+def select_compact_stress(log2_tokens=28, T=8192, reps=5):
+    """Selection, compaction and row packing on a stream long enough (2^28 tokens) for HBM
+    bandwidth, not launch latency, to be what is measured."""
+    import numpy as np
+    import torch
+    from paper_2603_06619_b200 import nat
+    from paper_2603_06619_b200 import workloads as wl
+    from paper_2603_06619_b200.step import NatStep
+
+    n_tot = 1 << log2_tokens
+    B = n_tot // T
+    G = 8
+    P = B // G
+    cu = torch.arange(0, n_tot + 1, T, dtype=torch.int32, device="cuda")
+    st = NatStep(P, G, 64, 512, torch.float32, n_tot, want_grads=False)
+    peaks, kind = load_peaks()
+    hbm = peaks["hbm_gbs"]
+    out = [f"N_tot = 2^{log2_tokens} tokens, B = {B} responses of {T}; mean of {reps} calls; "
+           f"HBM peak {hbm:.0f} GB/s ({kind}).", "",
+           "| call | selected fraction | ms | algorithmic bytes | GB/s | of HBM peak |",
+           "|---|---|---|---|---|---|"]
+
+    def row(label, frac, ms, what, nbytes):
+        out.append(f"| {label} | {frac} | {ms:.3f} | {what} | {nbytes / ms / 1e6:.0f} | "
+                   f"{nbytes / ms / 1e6 / hbm:.3f} |")
+
+    for label, kw in (("URS p=0.5", dict(mode="urs", p=0.5)), ("RPC C=100", dict(mode="rpc", min_cut=100))):
+        ms = _time(lambda: st.select(cu, seed=1, **kw), reps)
+        st.compact(cu)
+        frac = int(st.n_sel.item()) / n_tot
+        row(f"nat_select {label}", f"{frac:.3f}", ms, "5 B/token (mask + pi written)", 5.0 * n_tot)
+        msc = _time(lambda: st.compact(cu, from_mask=True), reps)
+        row(f"nat_compact after {label}", f"{frac:.3f}", msc,
+            "1 B/token read + 8 B per selected token written", (1.0 + 8.0 * frac) * n_tot)
+        if kw["mode"] == "rpc":
+            msp = _time(lambda: st.compact(cu), reps)
+            row(f"nat_compact_prefix after {label}", f"{frac:.3f}", msp,
+                "8 B per selected token written (the mask is not read)", 8.0 * frac * n_tot)
+    # a cut law given as masses: three reads of q, mask and pi written
+    q = torch.rand(n_tot, device="cuda") / T
+    ws = nat.alloc_workspace(nat.nat_select_cutlaw_workspace_bytes(B, n_tot), "cuda")
+    ms = _time(lambda: nat.nat_select_cutlaw(B, cu, n_tot, q, 1, 0, st.mask, st.pi, st.cut_len, ws),
+               reps)
+    row("nat_select_cutlaw (random law)", "-", ms,
+        "4 B/token read (the law) + 5 B/token written; executed: the law is read 3 times", 9.0 * n_tot)
+    del q
+    st.grpo_adv(torch.zeros(B, device="cuda"))
+    ms = _time(lambda: st.grpo_adv(torch.zeros(B, device="cuda")), reps)
+    out.append(f"| nat_grpo_adv ({P} groups of {G}) | - | {ms:.3f} | launch bound | - | - |")
+    del st
+    # packing of the selected rows: the Qwen3-8B-shaped batch's hidden states under RPC
+    w = wl.WORKLOADS["qwen3_8b"]
+    Tl = wl.make_lengths(w, 0)
+    cu2 = torch.from_numpy(wl.cu_from_lengths(Tl)).cuda()
+    n2 = int(Tl.sum())
+    st2 = NatStep(w.P, w.G, 64, 512, torch.float32, n2, want_grads=False)
+    st2.select(cu2, "rpc", min_cut=100, seed=0)
+    st2.compact(cu2)
+    n_sel = int(st2.n_sel.item())
+    x = torch.randn(n2, w.d, device="cuda").to(torch.bfloat16)
+    packed = torch.empty_like(x)
+    full = torch.empty_like(x)
+    rowb = w.d * 2
+    ms = _time(lambda: nat.nat_gather_rows(x, st2.sel_idx, st2.n_sel, n2, packed), reps)
+    row(f"nat_gather_rows ({n_sel} of {n2} rows of {rowb} B)", f"{n_sel / n2:.3f}", ms,
+        "row read + row written", 2.0 * n_sel * rowb)
+    ms = _time(lambda: nat.nat_scatter_rows(packed, st2.sel_idx, st2.n_sel, n2, n2, full), reps)
+    row(f"nat_scatter_rows (same, into {n2} zeroed rows)", f"{n_sel / n2:.3f}", ms,
+        "row read + row written + zero fill", 2.0 * n_sel * rowb + 1.0 * n2 * rowb)
+    return "\n".join(out)
+
+
+def ceiling(base, rows=32768, seconds=4.0):
+    """Per contraction: TFLOP/s of the loss kernels and of the library GEMM (torch.matmul) on
+    the same shapes and operand values, each measured inside a loop that runs for `seconds`
+    under the power cap.  The library is called here only, never on the product path."""
+    import torch
+    from paper_2603_06619_b200 import nat
+    from paper_2603_06619_b200 import workloads as wl
+    from paper_2603_06619_b200.step import NatStep
+
+    T = rows // base.G
+    w = wl.variant(base, P=1, sel_mode="urs", p=1.0, length_law="uniform", len_lo=T, len_hi=T)
+    batch = wl.make_batch(w, seed=0, device="cuda")
+    st = NatStep(w.P, w.G, w.d, w.V, torch.bfloat16, batch["n_tot"])
+    cu = batch["cu_seqlens"]
+    st.grpo_adv(batch["rewards"])
+    st.select(cu, "urs", p=1.0)
+    st.compact(cu)
+    n = int(st.n_sel.item())
+    args = (batch["hidden"], batch["W"], batch["targets"], batch["old_logp"], cu)
+    ms_call = _time(lambda: st.loss_fwd_bwd(*args), 2)
+    calls = max(2, int(seconds * 1e3 / ms_call))
+    sampler = ClockSampler(torch.cuda.current_device())
+    for _ in range(calls // 2):
+        st.loss_fwd_bwd(*args)
+    sampler.start()
+    nat.nat_trace_begin()
+    for _ in range(calls - calls // 2):
+        st.loss_fwd_bwd(*args)
+    tr = nat.nat_trace_end()
+    torch.cuda.synchronize()
+    ours_clk = sampler.stop()
+    assert st.status() & ~4 == 0
+    traced = calls - calls // 2
+    flop = 2.0 * n * w.d * w.V
+    ours = {k: flop / (tr[k][0] / traced * 1e-3) / 1e12 for k in ("e", "dh", "dw")}
+
+    # the same three products by the library, chunk by chunk, on the same values
+    chunk = 8192
+    W = batch["W"]
+    Hc = batch["hidden"][:chunk]
+    S = (Hc @ W.t()).float()
+    E = torch.exp(S - S[:, :256].max(dim=1, keepdim=True).values).to(torch.bfloat16)
+    del S
+    Hs = (Hc.float() * (-1e-4 / E.float().sum(dim=1, keepdim=True))).to(torch.bfloat16)
+    Et = E.t()
+    Wt = W.t()
+    out_s = torch.empty(chunk, w.V, dtype=torch.bfloat16, device="cuda")
+    out_h = torch.empty(chunk, w.d, dtype=torch.bfloat16, device="cuda")
+    out_w = torch.empty(w.V, w.d, dtype=torch.bfloat16, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+
+    def lib_chunk(record):
+        if record:
+            ev[0].record()
+        torch.matmul(Hc, Wt, out=out_s)
+        if record:
+            ev[1].record()
+        torch.matmul(E, W, out=out_h)
+        if record:
+            ev[2].record()
+        torch.matmul(Et, Hs, out=out_w)
+        if record:
+            ev[3].record()
+
+    ms_chunk = _time(lambda: lib_chunk(False), 4)
+    reps = max(4, int(seconds * 1e3 / ms_chunk))
+    for _ in range(reps // 2):
+        lib_chunk(False)
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    sums = [0.0, 0.0, 0.0]
+    for _ in range(reps - reps // 2):
+        lib_chunk(True)
+        torch.cuda.synchronize()
+        for j in range(3):
+            sums[j] += ev[j].elapsed_time(ev[j + 1])
+    lib_clk = sampler.stop()
+    timed = reps - reps // 2
+    cflop = 2.0 * chunk * w.d * w.V
+    lib = {k: cflop / (sums[j] / timed * 1e-3) / 1e12 for j, k in enumerate(("e", "dh", "dw"))}
+    peaks, kind = load_peaks()
+    label = {"e": "S = Hc W^T (kE: + exp, row sums, bf16 store)",
+             "dh": "dH = E W (kDh: + row factor, one-hot term)",
+             "dw": "dW += E^T Hs (kDw: fp32 accumulation into dW)"}
+    out = [f"{n} rows of the {base.name} head (d = {w.d}, V = {w.V}); each side looped for about "
+           f"{seconds:.0f} s, second half timed; library = torch.matmul, bf16 output, no "
+           f"accumulation; peaks {kind}: sustained {peaks['bf16_tflops_sustained']:.0f} TFLOP/s.", "",
+           "| contraction | loss kernel TFLOP/s | library GEMM TFLOP/s | ratio |", "|---|---|---|---|"]
+    for k in ("e", "dh", "dw"):
+        out.append(f"| {label[k]} | {ours[k]:.0f} | {lib[k]:.0f} | {ours[k] / lib[k]:.3f} |")
+    tot_o = 3.0 / sum(1.0 / ours[k] for k in ours)
+    tot_l = 3.0 / sum(1.0 / lib[k] for k in lib)
+    out.append(f"| all three (harmonic mean) | {tot_o:.0f} | {tot_l:.0f} | {tot_o / tot_l:.3f} |")
+    out += ["", f"SM clock / board power while looping (medians): loss kernels "
+            f"{ours_clk['sm_mhz']} MHz / {ours_clk['power_w']} W, library {lib_clk['sm_mhz']} MHz / "
+            f"{lib_clk['power_w']} W."]
+    return "\n".join(out)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="step",
+                    choices=["step", "sweep", "stress", "ceiling", "source-hash"])
     ap.add_argument("--workload", default="qwen3_8b")
+    ap.add_argument("--selection", default=None,
+                    help="override the workload's selection: urs:P, rpc:C or det:BETA")
+    ap.add_argument("--prompts", type=int, default=0,
+                    help="override the workload's number of prompts (a reduced case of the same "
+                         "head, e.g. for profiler captures)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=384,
                     help="selected rows the fp64 oracle evaluates per timed sample (about 15 s on 16 cores)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="N > 1: the ranks split ONE batch by prompt groups (global batch size in "
+                         "the weights, global response index in the selection) and all-reduce "
+                         "loss and dW every step; strong scaling")
     ap.add_argument("--allreduce-dw", action="store_true",
-                    help="N > 1: sum loss and dW over the ranks inside every step (the exchange of "
-                         "a data-parallel trainer); off by default: ranks then run independent "
-                         "batches with no collective")
+                    help="N > 1, independent batches: also sum loss and dW over the ranks inside "
+                         "every step (timing of the exchange only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-other-route", action="store_true",
                     help="do not also time the route that was not selected")
+    ap.add_argument("--only-steps", action="store_true",
+                    help="run the warm-up and the timed steps and nothing else (no per-kernel "
+                         "trace, other route, end-to-end or CPU legs): the case to put under a profiler")
     ap.add_argument("--route", default="single", choices=["single", "two"],
                     help="single: nat_policy_loss_fwd_bwd; two: forward then backward calls")
+    ap.add_argument("--reps", type=int, default=2, help="calls per point (sweep, stress)")
+    ap.add_argument("--log2-tokens", type=int, default=28, help="stream length of --mode stress")
     args = ap.parse_args()
-    from paper_2603_06619_b200 import workloads as wl
-    w = wl.WORKLOADS[args.workload]
+    if args.mode == "source-hash":
+        print(kernel_source_hash())
+        return
+    if args.impl == "ours" and args.mode == "step" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args, sys.argv[1:]))
+    w = pick_workload(args)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.mode == "sweep":
+        from paper_2603_06619_b200 import build as _build
+        _build.build()
+        print(fraction_sweep(w, reps=args.reps, seed=args.seed))
+    elif args.mode == "stress":
+        from paper_2603_06619_b200 import build as _build
+        _build.build()
+        print(select_compact_stress(log2_tokens=args.log2_tokens, reps=max(args.reps, 5)))
+    elif args.mode == "ceiling":
+        from paper_2603_06619_b200 import build as _build
+        _build.build()
+        print(ceiling(w))
     else:
         run_ours(args, w)
 

@@ -4,8 +4,10 @@ This module only draws inputs (lengths, hidden states, LM-head weights,
 targets, rewards, behaviour-policy log-probs).  It holds none of the method's
 arithmetic: selection, weighting, the surrogate and its gradients live in the
 CUDA library (and, separately, in the test oracle).  The one derived input,
-``old_logp``, is a library log-softmax of the drawn logits plus noise; it is an
-input like any other and both sides receive the same bytes.
+``old_logp``, is a library log-softmax of the drawn logits plus noise (torch's
+matmul and logsumexp: the only place in the package where a library GEMM runs,
+and only to make an input); it is an input like any other and both sides
+receive the same bytes.
 
 Shapes follow the paper's training recipe (8 rollouts per prompt, responses up
 to 8192 tokens for Qwen3-8B, Appendix C) and the Qwen3 head sizes
@@ -117,12 +119,15 @@ def library_logp(hidden, W, targets, rows_per_chunk=4096):
     return out
 
 
-def make_batch(w: Workload, seed: int = 0, device="cpu", lengths=None):
+def make_batch(w: Workload, seed: int = 0, device="cpu", lengths=None, W_seed=None):
     """Draw one batch.  Returns a dict of torch tensors on ``device``:
 
     lengths/cu_seqlens int32, hidden [N_tot, d], W [V, d] (dtype of the
     workload), targets int32 [N_tot], rewards float32 [B], old_logp float32
     [N_tot].
+
+    ``W_seed``: draw W from a generator of its own with this seed, so that data-parallel
+    ranks that draw different shards (different ``seed``) hold the same replicated W.
     """
     T = make_lengths(w, seed) if lengths is None else np.asarray(lengths, dtype=np.int32)
     cu = cu_from_lengths(T)
@@ -132,7 +137,11 @@ def make_batch(w: Workload, seed: int = 0, device="cpu", lengths=None):
     g.manual_seed(1000003 * seed + 17)
     dt = _torch_dtype(w)
     hidden = torch.randn(n_tot, w.d, generator=g, device=dev, dtype=torch.float32).to(dt)
-    W = (torch.randn(w.V, w.d, generator=g, device=dev, dtype=torch.float32) * w.w_scale).to(dt)
+    gW = g
+    if W_seed is not None:
+        gW = torch.Generator(device=dev)
+        gW.manual_seed(1000003 * int(W_seed) + 29)
+    W = (torch.randn(w.V, w.d, generator=gW, device=dev, dtype=torch.float32) * w.w_scale).to(dt)
     targets = torch.randint(0, w.V, (n_tot,), generator=g, device=dev, dtype=torch.int32)
     rewards = (torch.rand(w.B, generator=g, device=dev) < w.reward_p).float()
     noise = torch.randn(n_tot, generator=g, device=dev, dtype=torch.float32) * w.old_noise
