@@ -202,7 +202,8 @@ def select_cutlaw(cu_seqlens, q, *, seed=0, offset=0, resp_base=0):
     right after that token, q_i(l) up to a common factor per response.  With the fixed-point
     counts k of ``cutlaw_counts``:
         S_t  = sum_{l >= t} k_l                 (Eq. rpc-survival's suffix sum, exact integers)
-        pi_t = float32(double(S_t) / double(S_1))      so pi_1 = 1, pi non-increasing
+        pi_t = float32(double(S_t) * (1 / double(S_1)))   (the reciprocal once per response;
+               every operation IEEE round-to-nearest)  so pi_1 = 1, pi non-increasing
         u    = x1 2^32 + x0 from the Philox block with counter (0, resp_base + i, 3, offset_lo)
         r    = floor(u S_1 / 2^64)              uniform on {0 .. S_1 - 1} to within S_1 2^-64
         m_t  = [S_t > r]                        i.e. L_i = max{t : S_t > r}, Pr(L_i >= t) = S_t / S_1
@@ -239,7 +240,8 @@ def select_cutlaw(cu_seqlens, q, *, seed=0, offset=0, resp_base=0):
         r = (u * total) >> 64
         S64 = np.array(S, dtype=np.uint64)
         mask[lo:hi] = (S64 > np.uint64(r)).astype(np.uint8)
-        pi[lo:hi] = (S64.astype(np.float64) / np.float64(np.uint64(total))).astype(np.float32)
+        inv_total = np.float64(1.0) / np.float64(np.uint64(total))
+        pi[lo:hi] = (S64.astype(np.float64) * inv_total).astype(np.float32)
         cut_len[i] = int(mask[lo:hi].sum())
     return mask, pi, cut_len
 

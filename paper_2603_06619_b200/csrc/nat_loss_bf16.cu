@@ -86,6 +86,9 @@ struct TcParams {
   const float* mref;       // kE: per-row reference
   const float* row_scale;  // kDh: per-row factor on the accumulator (null = 1)
   int b_row0;              // kDw: first row of the B operand's tensor map for this launch
+  int k_splits;            // kDh: the K range (the vocabulary) is cut into this many units per
+                           //   output tile; above 1 the partial tiles are added into a float32
+                           //   scratch (mapC) and dh_finalize_kernel forms dHidden from it
   const int32_t* flag;     // predicate: the launch does nothing unless
   int run_if;              //   (*flag != 0) == run_if   (flag == null: always runs)
   int32_t* ovf;            // kE: set to 1 when the window is exceeded
@@ -97,7 +100,9 @@ struct Unit {
   int mb;      // block along the accumulator's M dimension
   int nt_lo;   // first and one-past-last block along N
   int nt_hi;
-  int sp;      // vocabulary split (kFwd, kDz)
+  int sp;      // vocabulary split (kFwd, kDz, kE)
+  int kb_lo;   // k-blocks of this unit: the whole K range, or one of k_splits parts of it (kDh)
+  int kb_hi;
 };
 
 struct Shape {
@@ -126,7 +131,7 @@ __device__ __forceinline__ Shape make_shape(const TcParams& p) {
   } else if (MODE == kDh) {
     s.mblocks = (rows + BMU - 1) / BMU;
     s.nblocks = (p.d + BN - 1) / BN;
-    s.n_units = s.mblocks * s.nblocks;
+    s.n_units = s.mblocks * s.nblocks * p.k_splits;
     s.kb = (p.V + BK - 1) / BK;
   } else {
     s.mblocks = (p.V + BMU - 1) / BMU;
@@ -144,7 +149,14 @@ template <int MODE, int CTAS, int SUBS>
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Shape& s, int u) {
   constexpr int kGroup = kGroupRows / (CTAS * SUBS);
   Unit w;
+  w.kb_lo = 0;
+  w.kb_hi = s.kb;
   if (MODE == kFwd || MODE == kDz || MODE == kE) {
+    // kE: one vocabulary tile per split, so a unit is one tile and the CTA pairs, which take
+    // units round-robin, work on the same few vocabulary tiles at any time (a W tile is
+    // fetched from DRAM once and found in L2 by the other row blocks of the group) without
+    // any pair waiting for another.  The group (4096 rows) keeps the rows' operand blocks
+    // (32 MB at d = 4096) resident in L2 next to the W tiles and the streaming stores.
     const int per_group = kGroup * p.n_splits;
     const int grp = u / per_group;
     const int rem = u - grp * per_group;
@@ -154,6 +166,20 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Shape& s, i
     w.mb = grp * kGroup + (rem - w.sp * rows_in_group);
     w.nt_lo = (int)(((long long)w.sp * s.nblocks) / p.n_splits);
     w.nt_hi = (int)(((long long)(w.sp + 1) * s.nblocks) / p.n_splits);
+  } else if (MODE == kDh) {
+    // (K part, row block, column block), the column block varying fastest: the pairs in
+    // flight work on one K part, i.e. on the same half of W and the same few slabs of the
+    // numerators (measured 2 % faster per step than taking the parts of a tile in turn)
+    w.sp = 0;
+    const int per_ks = s.mblocks * s.nblocks;
+    const int ks = u / per_ks;
+    const int rem = u - ks * per_ks;
+    w.mb = rem / s.nblocks;
+    w.nt_lo = rem - w.mb * s.nblocks;
+    w.nt_hi = w.nt_lo + 1;
+    const int per = (s.kb + p.k_splits - 1) / p.k_splits;
+    w.kb_lo = ks * per;
+    w.kb_hi = w.kb_lo + per < s.kb ? w.kb_lo + per : s.kb;
   } else {
     w.sp = 0;
     w.mb = u / s.nblocks;
@@ -267,7 +293,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
       for (int u = unit0; ok && u < shape.n_units; u += unit_stride) {
         const Unit w = decode_unit<MODE, CTAS, SUBS>(p, shape, u);
         for (int nt = w.nt_lo; ok && nt < w.nt_hi; ++nt) {
-          if ((MODE == kFwd || MODE == kDz || MODE == kE) && rank == 0 && p.progress != nullptr) {
+          if ((MODE == kFwd || MODE == kDz) && rank == 0 && p.progress != nullptr) {
             // Pacing.  The CTAs that sweep the same vocabulary split for different row
             // blocks share every W tile through L2 only while they stay within a few
             // tiles of each other; left alone they drift apart (nothing slows the one in
@@ -305,7 +331,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
               }
             }
           }
-          for (int kb = 0; kb < shape.kb; ++kb, ++it) {
+          for (int kb = w.kb_lo; kb < w.kb_hi; ++kb, ++it) {
             const int s = it % kNS;
             const uint32_t ph = (it / kNS) & 1u;
             if (!tc::mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -376,7 +402,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
           if (!tc::mbar_wait(&tempty_bar[acc], aph ^ 1u, abort_flag)) { ok = false; break; }
           tc::fence_after_sync();
           const uint32_t d_tmem = tmem_base + acc * SUBS * BN;
-          for (int kb = 0; kb < shape.kb; ++kb, ++it) {
+          for (int kb = w.kb_lo; kb < w.kb_hi; ++kb, ++it) {
             const int s = it % kNS;
             const uint32_t ph = (it / kNS) & 1u;
             if (!tc::mbar_wait(&full_bar[s], ph, abort_flag)) { ok = false; break; }
@@ -400,9 +426,9 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                   kBmn ? tc::smem_desc_sw128(b_base + kk * 2048, kBoxBytes, 1024)
                        : tc::smem_desc_sw128(b_base + kk * 32, 16, 1024);
               if (CTAS == 2)
-                tc::umma_bf16_pair(d_tmem + sub * BN, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+                tc::umma_bf16_pair(d_tmem + sub * BN, adesc, bdesc, kIdesc, (kb > w.kb_lo || kk > 0) ? 1u : 0u);
               else
-                tc::umma_bf16(d_tmem + sub * BN, adesc, bdesc, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+                tc::umma_bf16(d_tmem + sub * BN, adesc, bdesc, kIdesc, (kb > w.kb_lo || kk > 0) ? 1u : 0u);
               }
             }
             if (CTAS == 2) tc::umma_commit_pair(&empty_bar[s], 3);
@@ -610,6 +636,22 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
               if (col0 + 8 * g8 < ncols)
                 *reinterpret_cast<uint4*>(dst + 8 * g8) = make_uint4(
                     packed[4 * g8], packed[4 * g8 + 1], packed[4 * g8 + 2], packed[4 * g8 + 3]);
+          } else if (MODE == kDh && SUBS == 2 && p.k_splits > 1) {
+            // partial tile of a K part: added into the float32 scratch through the warp's
+            // staging block (TMA reduction), like kDw below; rows past the chunk are clipped
+            uint8_t* stage = staging + (warp - 2) * 4096;
+            if (lane == 0) tc::bulk_wait_read_all();
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<float4*>(stage + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                  make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tc::tma_reduce_add_2d(&mapC, stage, col0, lrow);
+              tc::bulk_commit();
+            }
           } else if (MODE == kDh) {
             if (row_ok) {
               const int k = p.row0 + lrow;
@@ -676,9 +718,9 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
         if (zt_found) p.zt[k] = zt_val;
       }
       if (MODE == kE && ok && row_ok) {
-        const int k = p.row0 + lrow;
-        p.part_s[(size_t)w.sp * p.cap_pad + k] = s_run;
-        if (zt_found) p.zt[k] = zt_val;
+        // one partial row sum per vocabulary tile, local to the chunk: [tile][row in chunk]
+        p.part_s[(size_t)w.sp * p.cap_pad + lrow] = s_run;
+        if (zt_found) p.zt[p.row0 + lrow] = zt_val;
         if (over) *p.ovf = 1;
       }
     }
@@ -760,31 +802,41 @@ __global__ void fwd_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_se
 // sums of E = exp(z - mref): lse = mref + log sum, logp, loss term, g, the row factor
 // c = -g / sum, and Hs[row - row0, :] = c * Hc[row, :].  Rows past the last selected
 // token are zero-filled in Hs.
-__global__ void fused_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_sel, int cap,
-                                      int row0, int chunk_rows, int n_splits, int cap_pad,
-                                      const float* __restrict__ mref,
-                                      const float* __restrict__ part_s,
-                                      const float* __restrict__ zt, const float* __restrict__ dloss,
-                                      float* __restrict__ logp, float* __restrict__ lse,
-                                      float* __restrict__ term, float* __restrict__ g_out,
-                                      float* __restrict__ cs, const __nv_bfloat16* __restrict__ Hc,
-                                      __nv_bfloat16* __restrict__ Hs, int d,
-                                      const int32_t* __restrict__ flag) {
+__global__ void __launch_bounds__(128)
+fused_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_sel, int cap, int row0,
+                      int chunk_rows, int n_parts, const float* __restrict__ mref,
+                      const float* __restrict__ part_s, const float* __restrict__ zt,
+                      const float* __restrict__ dloss, float* __restrict__ logp,
+                      float* __restrict__ lse, float* __restrict__ term, float* __restrict__ g_out,
+                      float* __restrict__ cs, const __nv_bfloat16* __restrict__ Hc,
+                      __nv_bfloat16* __restrict__ Hs, int d, const int32_t* __restrict__ flag) {
   if (predicate_off(flag, 0)) return;
   __shared__ float c_s;
+  __shared__ float warp_sum[4];
   int n = *n_sel;
   n = n < cap ? n : cap;
   const float dl = dloss ? *dloss : 1.f;
   const int vec = d / 8;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int r = blockIdx.x; r < chunk_rows; r += gridDim.x) {
     const int k = row0 + r;
     if (k >= n && r >= ((n - row0 + kRowPad - 1) / kRowPad) * kRowPad) break;  // beyond the tiles in use
     __syncthreads();
+    if (k < n) {
+      // the row's sum of numerators: one partial per vocabulary tile, [tile][row in chunk];
+      // every thread adds a strided share, then a fixed tree combines them
+      float part = 0.f;
+      for (int sp = threadIdx.x; sp < n_parts; sp += 128)
+        part += part_s[(size_t)sp * chunk_rows + r];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+      if (lane == 0) warp_sum[warp] = part;
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
       float cv = 0.f;
       if (k < n) {
-        float S = 0.f;
-        for (int sp = 0; sp < n_splits; ++sp) S += part_s[(size_t)sp * cap_pad + k];
+        const float S = (warp_sum[0] + warp_sum[1]) + (warp_sum[2] + warp_sum[3]);
         const float l = mref[k] + logf(S);
         const float lp = target_ok(c, k) ? zt[k] - l : __int_as_float(0x7FC00000);
         lse[k] = l;
@@ -816,6 +868,46 @@ __global__ void fused_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_
         }
         dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
       }
+    }
+  }
+}
+
+// dHidden of one row chunk from the float32 sums of the K parts (kDh with k_splits > 1):
+//   dH[k, :] = scale_k * acc[k - row0, :] + g_k W[y_k, :]   (one block per row).
+__global__ void __launch_bounds__(128)
+dh_finalize_kernel(const float* __restrict__ acc, const float* __restrict__ row_scale,
+                   const float* __restrict__ g, const __nv_bfloat16* __restrict__ W,
+                   const int32_t* __restrict__ targets, const int32_t* __restrict__ sel_idx,
+                   const int32_t* __restrict__ n_sel, int cap, int row0, int chunk_rows, int d,
+                   int V, __nv_bfloat16* __restrict__ dH, const int32_t* __restrict__ flag,
+                   int run_if) {
+  if (predicate_off(flag, run_if)) return;
+  int n = *n_sel;
+  n = n < cap ? n : cap;
+  const int vec = d / 8;
+  for (int r = blockIdx.x; r < chunk_rows; r += gridDim.x) {
+    const int k = row0 + r;
+    if (k >= n) break;
+    const float scale = row_scale ? row_scale[k] : 1.f;
+    const float gk = g[k];
+    int y = targets[sel_idx[k]];
+    if ((unsigned)y >= (unsigned)V) y = 0;  // such a token has g = 0
+    const float4* a = reinterpret_cast<const float4*>(acc + (size_t)r * d);
+    const uint4* wsrc = reinterpret_cast<const uint4*>(W + (size_t)y * d);
+    uint4* dst = reinterpret_cast<uint4*>(dH + (size_t)k * d);
+    for (int j = threadIdx.x; j < vec; j += blockDim.x) {
+      const float4 a0 = a[2 * j], a1 = a[2 * j + 1];
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const uint4 wv = __ldg(wsrc + j);
+      const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 w2 = *reinterpret_cast<const __nv_bfloat162*>(&ww[e]);
+        o[e] = pack_bf16(fmaf(gk, __low2float(w2), scale * av[2 * e]),
+                         fmaf(gk, __high2float(w2), scale * av[2 * e + 1]));
+      }
+      dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
     }
   }
 }
@@ -954,8 +1046,9 @@ onehot_apply_kernel(const __nv_bfloat16* __restrict__ Hc, const float* __restric
 // ------------------------------------------------------------- host side
 struct Layout {
   int cap_pad, n_tiles, n_splits, chunk_rows, n_chunks, ldz;
-  size_t off_term, off_g, off_zt, off_pm, off_ps, off_mref, off_cs, off_ovf, off_prog, off_ohc,
-      off_oho, off_ohl, off_ohs, off_hc, off_hs, off_dz, total;
+  int dh_splits;  // K parts of the dHidden contraction (1: direct epilogue)
+  size_t off_term, off_g, off_zt, off_pm, off_ps, off_pe, off_mref, off_cs, off_ovf, off_prog,
+      off_ohc, off_oho, off_ohl, off_ohs, off_hc, off_hs, off_dhacc, off_dz, total;
 };
 
 // Number of vocabulary splits.  A work unit of the vocabulary sweeps is (block of rows,
@@ -986,6 +1079,28 @@ int pick_splits(int n_tiles, int m_units, int slots) {
 
 int pair_slots();
 
+// Number of K parts of the dHidden contraction.  Its work units are (512-row block,
+// 256-column block) tiles over the whole vocabulary as K: few and long (256 for a full chunk
+// at d = 4096), so the last round of the CTA pairs is mostly empty.  Cutting K into parts
+// multiplies the units; the parts of a tile meet in a float32 scratch.  The smallest count
+// that fills the rounds to 95 % is taken (1 when CTA pairs are not available).
+int pick_k_splits(int tiles, int kb, int slots) {
+  if (slots <= 0 || tiles <= 0) return 1;
+  int best = 1;
+  double best_eff = 0.0;
+  for (int s = 1; s <= 8; ++s) {
+    if (s > 1 && kb / s < 64) break;
+    const long long units = (long long)tiles * s;
+    const double eff = (double)units / (double)(((units + slots - 1) / slots) * slots);
+    if (eff > best_eff + 1e-9) {
+      best = s;
+      best_eff = eff;
+    }
+    if (eff >= 0.95) return s;
+  }
+  return best;
+}
+
 // Hidden sizes from which the single-pass sweep uses 512-row work units (see launch_tc).
 bool wide_sweep(int d) { return d >= 2048; }
 
@@ -999,6 +1114,8 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   L.n_splits = pick_splits(L.n_tiles, L.chunk_rows / (wide_sweep(p.d) ? 512 : 256), pair_slots());
   L.n_chunks = (L.cap_pad + L.chunk_rows - 1) / L.chunk_rows;
   L.ldz = (p.V + 63) / 64 * 64;
+  L.dh_splits = pick_k_splits((L.chunk_rows / 512) * ((p.d + BN - 1) / BN), (p.V + BK - 1) / BK,
+                              pair_slots());
   size_t off = sizeof(WorkspaceHead);
   auto take = [&](size_t bytes) {
     const size_t o = off;
@@ -1010,6 +1127,7 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   L.off_zt = take(sizeof(float) * L.cap_pad);
   L.off_pm = take(sizeof(float) * (size_t)L.cap_pad * L.n_splits);
   L.off_ps = take(sizeof(float) * (size_t)L.cap_pad * L.n_splits);
+  L.off_pe = take(sizeof(float) * (size_t)L.chunk_rows * L.n_tiles);
   L.off_mref = take(sizeof(float) * L.cap_pad);
   L.off_cs = take(sizeof(float) * L.cap_pad);
   L.off_ovf = take(sizeof(int32_t) * L.n_chunks);
@@ -1021,6 +1139,7 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   off = align_up(off, 1024);
   L.off_hc = take(sizeof(__nv_bfloat16) * (size_t)L.cap_pad * p.d);
   L.off_hs = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * p.d);
+  L.off_dhacc = take(L.dh_splits > 1 ? sizeof(float) * (size_t)L.chunk_rows * p.d : 0);
   L.off_dz = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * L.ldz);
   L.total = off;
   return L;
@@ -1234,7 +1353,7 @@ int launch_tc(const CUtensorMap& a, const CUtensorMap& b1, const CUtensorMap& b2
 
 struct Ws {
   WorkspaceHead* head;
-  float *term, *g, *zt, *pm, *ps, *mref, *cs;
+  float *term, *g, *zt, *pm, *ps, *pe, *mref, *cs, *dhacc;
   int32_t* ovf;
   unsigned long long* prog;
   int32_t *oh_count, *oh_off, *oh_list, *oh_sorted;  // grouping of the tokens by target
@@ -1250,6 +1369,8 @@ Ws carve(void* ws, const Layout& L) {
   w.zt = reinterpret_cast<float*>(b + L.off_zt);
   w.pm = reinterpret_cast<float*>(b + L.off_pm);
   w.ps = reinterpret_cast<float*>(b + L.off_ps);
+  w.pe = reinterpret_cast<float*>(b + L.off_pe);
+  w.dhacc = reinterpret_cast<float*>(b + L.off_dhacc);
   w.mref = reinterpret_cast<float*>(b + L.off_mref);
   w.cs = reinterpret_cast<float*>(b + L.off_cs);
   w.ovf = reinterpret_cast<int32_t*>(b + L.off_ovf);
@@ -1290,6 +1411,7 @@ TcParams base_params(const LossArgs& a, const Layout& L, const Ws& w) {
   p.mref = w.mref;
   p.row_scale = nullptr;
   p.b_row0 = 0;
+  p.k_splits = 1;
   p.flag = nullptr;
   p.run_if = 0;
   p.ovf = nullptr;
@@ -1311,6 +1433,7 @@ struct Maps {
   CUtensorMap hcK, wK, wK2, dzK, wMn, dzMn, hcMn, hsMn;  // wK2: 128-row boxes for CTA pairs
   CUtensorMap dzSt;  // the numerator scratch as a store target: 64 columns x 32 rows
   CUtensorMap dwRed;  // dW as a reduction target (valid only when the call has a dW)
+  CUtensorMap dhAcc;  // the float32 scratch of the dHidden K parts as a reduction target
 };
 
 int encode_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
@@ -1327,8 +1450,16 @@ int encode_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
   if ((s = make_map(&m->dzSt, w.dz, a.p.V, L.chunk_rows, zpitch, 64, 32)) != NAT_OK) return s;
   m->dwRed = m->dzSt;
   if (a.dW != nullptr && (s = make_map_f32(&m->dwRed, a.dW, a.p.d, a.p.V)) != NAT_OK) return s;
+  m->dhAcc = m->dzSt;
+  if (L.dh_splits > 1 && (s = make_map_f32(&m->dhAcc, w.dhacc, a.p.d, L.chunk_rows)) != NAT_OK)
+    return s;
   return NAT_OK;
 }
+
+// dHidden of one row chunk: the contraction (in K parts when that fills the device better)
+// and, for K parts, the pass that forms dHidden from their float32 sum.
+int launch_dh(const LossArgs& a, const Layout& L, const Ws& w, const Maps& m, TcParams p,
+              const int32_t* flag, int run_if);
 
 // The tensor maps depend only on the operands' addresses and shapes, which a trainer keeps
 // from step to step, so the last few sets are remembered (encoding ten maps costs tens of
@@ -1374,6 +1505,30 @@ int finalize_grid(int rows) {
   return g < 1 ? 1 : (g > 1184 ? 1184 : g);
 }
 
+int launch_dh(const LossArgs& a, const Layout& L, const Ws& w, const Maps& m, TcParams p,
+              const int32_t* flag, int run_if) {
+  int s;
+  const int mb = L.chunk_rows / BM;
+  const int nb_d = (a.p.d + BN - 1) / BN;
+  p.flag = flag;
+  p.run_if = run_if;
+  const bool parts = L.dh_splits > 1 && pair_slots() > 0;
+  p.k_splits = parts ? L.dh_splits : 1;
+  if (parts)
+    NAT_CUDA(cudaMemsetAsync(w.dhacc, 0, sizeof(float) * (size_t)L.chunk_rows * a.p.d, a.stream));
+  if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, parts ? m.dhAcc : m.hcK, p, mb, nb_d * p.k_splits,
+                          a.stream)) != NAT_OK)
+    return s;
+  if (parts) {
+    dh_finalize_kernel<<<L.chunk_rows < 4096 ? L.chunk_rows : 4096, 128, 0, a.stream>>>(
+        w.dhacc, p.row_scale, w.g, reinterpret_cast<const __nv_bfloat16*>(a.W), a.targets,
+        a.sel_idx, a.n_sel, (int)a.cap, p.row0, L.chunk_rows, a.p.d, a.p.V,
+        reinterpret_cast<__nv_bfloat16*>(a.dHidden), flag, run_if);
+    NAT_LAUNCH_CHECK("dh_finalize_kernel");
+  }
+  return NAT_OK;
+}
+
 // The three two-pass backward launches for rows [row0, row0 + chunk_rows); `flag`
 // (may be null) predicates them on the chunk having left the single-pass window.
 int launch_two_pass_chunk(const LossArgs& a, const Layout& L, const Ws& w, const Maps& m,
@@ -1388,7 +1543,7 @@ int launch_two_pass_chunk(const LossArgs& a, const Layout& L, const Ws& w, const
   const int mb = L.chunk_rows / BM;
   const int nb_d = (a.p.d + BN - 1) / BN;
   if ((s = launch_tc<kDz>(m.hcK, m.wK, m.wK2, m.hcK, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
-  if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, m.hcK, p, mb, nb_d, a.stream)) != NAT_OK) return s;
+  if ((s = launch_dh(a, L, w, m, p, flag, 1)) != NAT_OK) return s;
   return launch_tc<kDw>(m.dzMn, m.hcMn, m.hcMn, m.dwRed, p, (a.p.V + BM - 1) / BM, nb_d, a.stream);
 }
 
@@ -1495,17 +1650,27 @@ int loss_bf16_fwd_bwd(const LossArgs& a) {
       p.row0 = row0;
       p.chunk_rows = L.chunk_rows;
       p.ovf = ovf;
-      if ((s = launch_tc<kE>(m.hcK, m.wK, m.wK2, m.dzSt, p, mb, L.n_splits, a.stream)) != NAT_OK) return s;
+      {
+        // one work unit per (row block, vocabulary tile); partial row sums per tile, local
+        // to the chunk
+        TcParams pe = p;
+        pe.n_splits = L.n_tiles;
+        pe.part_s = w.pe;
+        pe.cap_pad = L.chunk_rows;
+        pe.progress = nullptr;
+        if ((s = launch_tc<kE>(m.hcK, m.wK, m.wK2, m.dzSt, pe, mb, L.n_tiles, a.stream)) != NAT_OK)
+          return s;
+      }
       fused_finalize_kernel<<<L.chunk_rows < 2048 ? L.chunk_rows : 2048, 128, 0, a.stream>>>(
-          c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_splits, L.cap_pad, w.mref, w.ps, w.zt,
-          a.dloss, a.logp, a.lse, w.term, w.g, w.cs, w.hc, w.hs, a.p.d, ovf);
+          c, a.n_sel, (int)a.cap, row0, L.chunk_rows, L.n_tiles, w.mref, w.pe, w.zt, a.dloss,
+          a.logp, a.lse, w.term, w.g, w.cs, w.hc, w.hs, a.p.d, ovf);
       NAT_LAUNCH_CHECK("fused_finalize_kernel");
       p.ovf = nullptr;
-      p.flag = ovf;
-      p.run_if = 0;
       p.row_scale = w.cs;
       p.b_row0 = 0;  // Hs is local to the chunk
-      if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, m.hcK, p, mb, nb_d, a.stream)) != NAT_OK) return s;
+      if ((s = launch_dh(a, L, w, m, p, ovf, 0)) != NAT_OK) return s;
+      p.flag = ovf;
+      p.run_if = 0;
       if ((s = launch_tc<kDw>(m.dzMn, m.hsMn, m.hsMn, m.dwRed, p, (a.p.V + BM - 1) / BM, nb_d,
                               a.stream)) != NAT_OK)
         return s;

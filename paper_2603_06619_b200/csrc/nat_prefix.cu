@@ -129,7 +129,7 @@ prefix_write_kernel(int B, const int32_t* __restrict__ cu, const int32_t* __rest
 __device__ __forceinline__ unsigned long long cutlaw_count(float q) {
   if (!(q > 0.f)) return 0ull;
   // the product is exact (a power-of-two scaling) and below 2^32 unless q >= 1
-  return q >= 1.f ? (1ull << 32) : (unsigned long long)__fmul_rn(q, 4294967296.f);
+  return q >= 1.f ? (1ull << 32) : (unsigned long long)__float2uint_rz(__fmul_rn(q, 4294967296.f));
 }
 
 __device__ __forceinline__ void load_counts(const float* __restrict__ q, int64_t n0, int64_t n_tot,
@@ -235,7 +235,7 @@ cutlaw_starts_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
                      unsigned long long* __restrict__ rstart) {
   __shared__ unsigned long long warp_tot[kSelThreads / 32];
   __shared__ unsigned long long thread_excl[kSelThreads];
-  __shared__ unsigned long long k_s[kSelBlockTokens];
+  __shared__ unsigned long long k_s[kSelThreads * kPiPad];  // 17 slots per thread: no bank conflicts
   __shared__ int first_s;
   const int64_t chunk0 = (int64_t)blockIdx.x * kSelBlockTokens;
   const int64_t chunk_end = min(chunk0 + (int64_t)kSelBlockTokens, n_tot);
@@ -261,7 +261,7 @@ cutlaw_starts_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
 #pragma unroll
   for (int j = 0; j < kTokPerThread; ++j) {
     s += k[j];
-    k_s[threadIdx.x * kTokPerThread + j] = k[j];
+    k_s[threadIdx.x * kPiPad + j] = k[j];
   }
   unsigned long long total;
   const unsigned long long excl = block_excl_scan(s, warp_tot, &total);
@@ -277,7 +277,7 @@ cutlaw_starts_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
       const int rel = (int)(n - chunk0);
       const int t = rel / kTokPerThread, j = rel % kTokPerThread;
       unsigned long long g = base + thread_excl[t];
-      for (int e = 0; e < j; ++e) g += k_s[t * kTokPerThread + e];
+      for (int e = 0; e < j; ++e) g += k_s[t * kPiPad + e];
       rstart[i] = g;
     }
   }
@@ -331,14 +331,14 @@ cutlaw_final_kernel(CutConst c, int B, const int32_t* __restrict__ cu, int64_t n
     int i = owner_between(cu, range_s[0], range_s[1], n0);
     int64_t start = cu[i], end = cu[i + 1];
     unsigned long long g0 = 0, S1 = 0, r = 0;
-    double inv_den = 1.0;
+    double inv_total = 1.0;
     auto enter_response = [&]() {
       g0 = rstart[i];
       S1 = rstart[i + 1] - g0;
       const Philox4 x = philox4x32_10(0u, c.resp_base + (uint32_t)i, 3u, c.off_lo, c.k0, c.k1);
       const unsigned long long u = ((unsigned long long)x.y << 32) | (unsigned long long)x.x;
       r = __umul64hi(u, S1);
-      inv_den = __ull2double_rn(S1);
+      inv_total = __drcp_rn(__ull2double_rn(S1));
     };
     enter_response();
     alignas(16) uint8_t m[kTokPerThread];
@@ -363,7 +363,7 @@ cutlaw_final_kernel(CutConst c, int B, const int32_t* __restrict__ cu, int64_t n
           const unsigned long long St = S1 - (G - g0);
           const bool keep = St > r;
           m[j] = keep ? 1 : 0;
-          pv = __double2float_rn(__ddiv_rn(__ull2double_rn(St), inv_den));
+          pv = __double2float_rn(__dmul_rn(__ull2double_rn(St), inv_total));
           // last kept token of the response: the next one is past the end or not kept
           if (keep && (n + 1 == end || !(St - k[j] > r))) cut_len[i] = (int32_t)(n - start) + 1;
         }
