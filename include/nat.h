@@ -143,15 +143,15 @@ int nat_select_survival(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, con
  * other than the uniform one).
  *   q float32 [n_tot]: the mass q_i(l) the law of token n's response puts on cutting right
  *   after that token, up to a common positive factor per response.  Masses enter in
- *   32-bit fixed point, k = floor(min(q, 1) 2^32) for q > 0 and 0 otherwise, so that every
- *   sum below is an exact 64-bit integer, independent of the order of summation:
+ *   32-bit fixed point, k = min(floor(q 2^32), 2^32 - 1) for q > 0 and 0 otherwise, so that
+ *   every sum below is an exact 64-bit integer, independent of the order of summation:
  *     S_t  = sum_{l >= t} k_l       (a scan over the packed stream on the device)
- *     pi_t = float32(double(S_t) * (1 / double(S_1))), every operation rounded to nearest:
- *            pi_1 = 1 and pi never increases, by construction; pi_t > 0 wherever the law
- *            still has mass at or after t
  *     u    = x1 2^32 + x0 of the Philox block with counter (0, resp_base + i, 3, offset_lo),
  *     r    = floor(u S_1 / 2^64),  m_t = [S_t > r]:  L_i = max{t : S_t > r},
- *            Pr(L_i >= t) = S_t / S_1 to within S_1 2^-64.
+ *            Pr(L_i >= t) = S_t / S_1 to within S_1 2^-64
+ *     pi_t = float32(double(S_t) * (1 / double(S_1))), every operation rounded to nearest:
+ *            pi_1 = 1 and pi never increases, by construction; pi_t > 0 wherever the law
+ *            still has mass at or after t.
  *   A response whose masses are all zero is kept whole with pi = 1.  Tokens after the
  *   last positive mass get pi = 0 and are never selected.
  * Outputs: mask uint8 [n_tot], pi float32 [n_tot], cut_len int32 [B].

@@ -182,16 +182,17 @@ def select_survival(cu_seqlens, surv, *, seed=0, offset=0, resp_base=0):
 
 
 def cutlaw_counts(q):
-    """Cut-law masses in 32-bit fixed point: k = floor(min(q, 1) * 2^32) for q > 0, else 0.
+    """Cut-law masses in 32-bit fixed point: k = min(floor(q * 2^32), 2^32 - 1) for q > 0,
+    else 0 (a negative or NaN mass counts as zero).
 
     The scaling by a power of two and the floor are exact, so the counts (and every sum of
     them, taken in 64-bit integers) do not depend on the order of evaluation.
     """
     q = np.asarray(q, dtype=np.float32)
     k = np.zeros(q.shape, dtype=np.uint64)
-    pos = q > 0                                     # NaN and negative masses count as zero
-    scaled = np.minimum(q[pos], np.float32(1.0)).astype(np.float64) * 4294967296.0
-    k[pos] = np.floor(scaled).astype(np.uint64)
+    pos = q > 0
+    scaled = np.floor(q[pos].astype(np.float64) * 4294967296.0)
+    k[pos] = np.minimum(scaled, 4294967295.0).astype(np.uint64)
     return k
 
 
@@ -202,11 +203,13 @@ def select_cutlaw(cu_seqlens, q, *, seed=0, offset=0, resp_base=0):
     right after that token, q_i(l) up to a common factor per response.  With the fixed-point
     counts k of ``cutlaw_counts``:
         S_t  = sum_{l >= t} k_l                 (Eq. rpc-survival's suffix sum, exact integers)
-        pi_t = float32(double(S_t) * (1 / double(S_1)))   (the reciprocal once per response;
-               every operation IEEE round-to-nearest)  so pi_1 = 1, pi non-increasing
         u    = x1 2^32 + x0 from the Philox block with counter (0, resp_base + i, 3, offset_lo)
         r    = floor(u S_1 / 2^64)              uniform on {0 .. S_1 - 1} to within S_1 2^-64
         m_t  = [S_t > r]                        i.e. L_i = max{t : S_t > r}, Pr(L_i >= t) = S_t / S_1
+        pi_t = float32(double(S_t) * (1 / double(S_1)))   (the reciprocal once per response;
+               every operation IEEE round-to-nearest)
+    so pi_1 = 1, pi never increases, and pi_t > 0 wherever the law still has mass at or
+    after t.
     A response whose counts are all zero is kept whole with pi = 1.
 
     Returns (mask uint8 [N_tot], pi float32 [N_tot], cut_len int32 [B]).

@@ -125,15 +125,23 @@ prefix_write_kernel(int B, const int32_t* __restrict__ cu, const int32_t* __rest
 }
 
 // ------------------------------------------------------------- cut laws
-// Fixed-point mass of one token: floor(min(q, 1) 2^32) for q > 0, else 0 (NaN counts as 0).
-__device__ __forceinline__ unsigned long long cutlaw_count(float q) {
-  if (!(q > 0.f)) return 0ull;
-  // the product is exact (a power-of-two scaling) and below 2^32 unless q >= 1
-  return q >= 1.f ? (1ull << 32) : (unsigned long long)__float2uint_rz(__fmul_rn(q, 4294967296.f));
+// Fixed-point mass of one token: min(floor(q 2^32), 2^32 - 1) for q > 0, else 0 (NaN and
+// negative masses count as 0).  Taken from the float's bits with integer operations only
+// (a float-to-integer conversion instruction runs at a sixteenth of their rate): q = m 2^e
+// with the 24-bit significand m, so floor(q 2^32) is m shifted by e + 32.
+__device__ __forceinline__ uint32_t cutlaw_count(float q) {
+  const uint32_t bits = __float_as_uint(q);
+  if (!(q > 0.f)) return 0u;                       // zero, negative, NaN
+  const int exp = (int)(bits >> 23);               // sign bit is clear here
+  if (exp >= 127) return 0xFFFFFFFFu;              // q >= 1 (infinity included)
+  if (exp == 0) return 0u;                         // subnormal: below 2^-126
+  const uint32_t m = (bits & 0x7FFFFFu) | 0x800000u;
+  const int sh = exp - 118;                        // (exp - 150) + 32; at most 8 here
+  return sh >= 0 ? m << sh : (sh > -24 ? m >> -sh : 0u);
 }
 
 __device__ __forceinline__ void load_counts(const float* __restrict__ q, int64_t n0, int64_t n_tot,
-                                            unsigned long long* k) {
+                                            uint32_t* k) {
   if (n0 + kTokPerThread <= n_tot) {
 #pragma unroll
     for (int v = 0; v < kTokPerThread / 4; ++v) {
@@ -145,7 +153,7 @@ __device__ __forceinline__ void load_counts(const float* __restrict__ q, int64_t
     }
   } else {
 #pragma unroll
-    for (int j = 0; j < kTokPerThread; ++j) k[j] = (n0 + j < n_tot) ? cutlaw_count(q[n0 + j]) : 0ull;
+    for (int j = 0; j < kTokPerThread; ++j) k[j] = (n0 + j < n_tot) ? cutlaw_count(q[n0 + j]) : 0u;
   }
 }
 
@@ -180,7 +188,7 @@ cutlaw_sum_kernel(const float* __restrict__ q, int64_t n_tot,
                   unsigned long long* __restrict__ chunk_sum) {
   __shared__ unsigned long long warp_tot[kSelThreads / 32];
   const int64_t n0 = (int64_t)blockIdx.x * kSelBlockTokens + (int64_t)threadIdx.x * kTokPerThread;
-  unsigned long long k[kTokPerThread];
+  uint32_t k[kTokPerThread];
   unsigned long long s = 0;
   if (n0 < n_tot) {
     load_counts(q, n0, n_tot, k);
@@ -225,22 +233,30 @@ cutlaw_scan_kernel(unsigned long long* __restrict__ chunk_sum, int n_chunks) {
   if (threadIdx.x == 0) chunk_sum[n_chunks] = carry;
 }
 
+struct CutConst {
+  uint32_t k0, k1, off_lo, resp_base;
+};
+
 // Pass 3: G[cu_i], the sum of all counts before the first token of response i, for every
 // response whose start lies in this chunk (the last chunk also takes the starts equal to
-// n_tot).  The chunk's counts are kept in shared memory so that a start in the middle of
-// a thread's 16 tokens can be resolved.
+// n_tot), and the response's 64-bit draw.  The chunk's counts are kept in shared memory so
+// that a start in the middle of a thread's 16 tokens can be resolved.
 __global__ void __launch_bounds__(kSelThreads)
-cutlaw_starts_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
+cutlaw_starts_kernel(CutConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
                      const float* __restrict__ q, const unsigned long long* __restrict__ chunk_off,
-                     unsigned long long* __restrict__ rstart) {
+                     unsigned long long* __restrict__ rstart,
+                     unsigned long long* __restrict__ udraw) {
   __shared__ unsigned long long warp_tot[kSelThreads / 32];
   __shared__ unsigned long long thread_excl[kSelThreads];
-  __shared__ unsigned long long k_s[kSelThreads * kPiPad];  // 17 slots per thread: no bank conflicts
+  __shared__ uint32_t k_s[kSelThreads * kPiPad];  // 17 slots per thread: no bank conflicts
   __shared__ int first_s;
   const int64_t chunk0 = (int64_t)blockIdx.x * kSelBlockTokens;
   const int64_t chunk_end = min(chunk0 + (int64_t)kSelBlockTokens, n_tot);
   if (threadIdx.x < 32) {  // first response whose start is >= chunk0
-    const int first_in = warp_upper_bound(cu, B, chunk0 - 1, 0);
+    int w0, first_in = 0;
+    const int64_t v = cu_window(cu, B, chunk0, n_tot, &w0);
+    if (!window_first(__ballot_sync(0xFFFFFFFFu, v >= chunk0), w0, &first_in))
+      first_in = warp_upper_bound(cu, B, chunk0 - 1, 0);
     if (threadIdx.x == 0) first_s = first_in;
   }
   __syncthreads();
@@ -253,7 +269,7 @@ cutlaw_starts_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
     if (c0 > chunk_end || (c0 == chunk_end && !last)) return;
   }
   const int64_t n0 = chunk0 + (int64_t)threadIdx.x * kTokPerThread;
-  unsigned long long k[kTokPerThread];
+  uint32_t k[kTokPerThread];
   unsigned long long s = 0;
 #pragma unroll
   for (int j = 0; j < kTokPerThread; ++j) k[j] = 0;
@@ -271,6 +287,10 @@ cutlaw_starts_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
   for (int i = first_in + (int)threadIdx.x; i <= B; i += kSelThreads) {
     const int64_t n = cu[i];
     if (n > chunk_end || (n == chunk_end && !last)) break;
+    if (i < B) {
+      const Philox4 x = philox4x32_10(0u, c.resp_base + (uint32_t)i, 3u, c.off_lo, c.k0, c.k1);
+      udraw[i] = ((unsigned long long)x.y << 32) | (unsigned long long)x.x;
+    }
     if (n == chunk_end) {  // the stream's end (only in the last chunk)
       rstart[i] = base + total;
     } else {
@@ -283,16 +303,23 @@ cutlaw_starts_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
   }
 }
 
-struct CutConst {
-  uint32_t k0, k1, off_lo, resp_base;
-};
+// double(x), correctly rounded.  Below 2^52 the value is exact and comes from one integer
+// OR and one addition (2^52 + x has x in its low significand bits); the conversion
+// instruction, which is slow, is left to the counts that large.
+__device__ __forceinline__ double u64_to_double(unsigned long long x) {
+  if (x < (1ull << 52))
+    return __dadd_rn(__longlong_as_double((long long)(0x4330000000000000ull | x)),
+                     -4503599627370496.0);
+  return __ull2double_rn(x);
+}
 
 // Pass 4: survival counts S_t = S_1 - (G[n] - G[cu_i]), the draw of each response, mask, pi
 // and the cut lengths.  One thread per 16 consecutive tokens.
-__global__ void __launch_bounds__(kSelThreads)
-cutlaw_final_kernel(CutConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
+__global__ void __launch_bounds__(kSelThreads, 4)
+cutlaw_final_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
                     const float* __restrict__ q, const unsigned long long* __restrict__ chunk_off,
-                    const unsigned long long* __restrict__ rstart, uint8_t* __restrict__ mask,
+                    const unsigned long long* __restrict__ rstart,
+                    const unsigned long long* __restrict__ udraw, uint8_t* __restrict__ mask,
                     float* __restrict__ pi, int32_t* __restrict__ cut_len) {
   __shared__ unsigned long long warp_tot[kSelThreads / 32];
   __shared__ float pi_s[kSelThreads * kPiPad];
@@ -317,7 +344,7 @@ cutlaw_final_kernel(CutConst c, int B, const int32_t* __restrict__ cu, int64_t n
   const int64_t n0 = nb0 + (int64_t)threadIdx.x * kTokPerThread;
   const bool active = n0 < n_tot;
   const int cnt = active ? (int)min((int64_t)kTokPerThread, n_tot - n0) : 0;
-  unsigned long long k[kTokPerThread];
+  uint32_t k[kTokPerThread];
   unsigned long long s = 0;
 #pragma unroll
   for (int j = 0; j < kTokPerThread; ++j) k[j] = 0;
@@ -330,51 +357,68 @@ cutlaw_final_kernel(CutConst c, int B, const int32_t* __restrict__ cu, int64_t n
     unsigned long long G = chunk_off[blockIdx.x] + excl;  // sum of all counts before token n0
     int i = owner_between(cu, range_s[0], range_s[1], n0);
     int64_t start = cu[i], end = cu[i + 1];
-    unsigned long long g0 = 0, S1 = 0, r = 0;
+    // St: the survival count of the current token, stepped down by its own count afterwards
+    unsigned long long S1 = 0, r = 0, St = 0;
     double inv_total = 1.0;
-    auto enter_response = [&]() {
-      g0 = rstart[i];
+    auto enter_response = [&](unsigned long long before) {  // `before`: counts preceding the token
+      const unsigned long long g0 = rstart[i];
       S1 = rstart[i + 1] - g0;
-      const Philox4 x = philox4x32_10(0u, c.resp_base + (uint32_t)i, 3u, c.off_lo, c.k0, c.k1);
-      const unsigned long long u = ((unsigned long long)x.y << 32) | (unsigned long long)x.x;
-      r = __umul64hi(u, S1);
-      inv_total = __drcp_rn(__ull2double_rn(S1));
+      St = S1 - (before - g0);
+      r = __umul64hi(udraw[i], S1);
+      inv_total = __drcp_rn(u64_to_double(S1));
     };
-    enter_response();
-    alignas(16) uint8_t m[kTokPerThread];
+    enter_response(G);
+    uint32_t bits = 0;
     float* pr = pi_s + threadIdx.x * kPiPad;
+    if (cnt == kTokPerThread && n0 + kTokPerThread <= end && S1 != 0ull) {
+      // the usual case: the thread's 16 tokens lie inside one response whose law has mass
 #pragma unroll
-    for (int j = 0; j < kTokPerThread; ++j) {
-      m[j] = 0;
-      float pv = 0.f;
-      if (j < cnt) {
-        const int64_t n = n0 + j;
-        while (n >= end) {  // skips empty responses too
-          ++i;
-          start = end;
-          end = cu[i + 1];
-          if (n < end) enter_response();
-        }
-        if (S1 == 0ull) {  // a law without mass: the response is kept whole
-          m[j] = 1;
-          pv = 1.f;
-          if (n + 1 == end) cut_len[i] = (int32_t)(end - start);
-        } else {
-          const unsigned long long St = S1 - (G - g0);
-          const bool keep = St > r;
-          m[j] = keep ? 1 : 0;
-          pv = __double2float_rn(__dmul_rn(__ull2double_rn(St), inv_total));
-          // last kept token of the response: the next one is past the end or not kept
-          if (keep && (n + 1 == end || !(St - k[j] > r))) cut_len[i] = (int32_t)(n - start) + 1;
-        }
+      for (int j = 0; j < kTokPerThread; ++j) {
+        bits |= (St > r ? 1u : 0u) << j;
+        pr[j] = __double2float_rn(__dmul_rn(u64_to_double(St), inv_total));
+        St -= k[j];
       }
-      pr[j] = pv;
-      G += k[j];
+      // the kept tokens are a prefix of the response; this thread holds its last one when
+      // some but not all of its tokens are kept, or all are and the next token (St is its
+      // survival count by now) is past the end or not kept
+      if (bits != 0u && (bits != 0xFFFFu || n0 + kTokPerThread == end || !(St > r)))
+        cut_len[i] = (int32_t)(n0 - start) + __popc(bits);
+    } else {
+#pragma unroll
+      for (int j = 0; j < kTokPerThread; ++j) {
+        float pv = 0.f;
+        if (j < cnt) {
+          const int64_t n = n0 + j;
+          if (n >= end) {
+            while (n >= end) {  // skips empty responses too
+              ++i;
+              start = end;
+              end = cu[i + 1];
+            }
+            enter_response(G);
+          }
+          if (S1 == 0ull) {  // a law without mass: the response is kept whole
+            bits |= 1u << j;
+            pv = 1.f;
+            if (n + 1 == end) cut_len[i] = (int32_t)(end - start);
+          } else {
+            const bool keep = St > r;
+            const unsigned long long next = St - k[j];  // survival count of the following token
+            bits |= (keep ? 1u : 0u) << j;
+            pv = __double2float_rn(__dmul_rn(u64_to_double(St), inv_total));
+            // last kept token of the response: the next one is past the end or not kept
+            if (keep && (n + 1 == end || !(next > r))) cut_len[i] = (int32_t)(n - start) + 1;
+            St = next;
+          }
+        }
+        pr[j] = pv;
+        G += k[j];
+      }
     }
     if (cnt == kTokPerThread) {
-      *reinterpret_cast<uint4*>(mask + n0) = *reinterpret_cast<const uint4*>(m);
+      *reinterpret_cast<uint4*>(mask + n0) = bits_to_bytes(bits);
     } else {
-      for (int j = 0; j < cnt; ++j) mask[n0 + j] = m[j];
+      for (int j = 0; j < cnt; ++j) mask[n0 + j] = (uint8_t)((bits >> j) & 1u);
     }
   }
   __syncthreads();
@@ -425,7 +469,7 @@ int nat_compact_prefix(int32_t B, const int32_t* cu_seqlens, int64_t n_tot,
 size_t nat_select_cutlaw_workspace_bytes(int32_t B, int64_t n_tot) {
   if (B < 0 || n_tot < 0) return 0;
   const int64_t chunks = (n_tot + nat::kSelBlockTokens - 1) / nat::kSelBlockTokens;
-  return nat::align_up((size_t)(chunks + 1) * 8, 256) + nat::align_up((size_t)(B + 1) * 8, 256);
+  return nat::align_up((size_t)(chunks + 1) * 8, 256) + 2 * nat::align_up((size_t)(B + 1) * 8, 256);
 }
 
 int nat_select_cutlaw(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const float* q,
@@ -452,6 +496,7 @@ int nat_select_cutlaw(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const
   unsigned long long* chunk_off = reinterpret_cast<unsigned long long*>(workspace);
   unsigned long long* rstart = reinterpret_cast<unsigned long long*>(
       reinterpret_cast<char*>(workspace) + align_up((size_t)(n_chunks + 1) * 8, 256));
+  unsigned long long* udraw = rstart + align_up((size_t)(B + 1) * 8, 256) / 8;
   NAT_CUDA(cudaMemsetAsync(cut_len, 0, sizeof(int32_t) * (size_t)B, stream));
   if (n_chunks == 0) return NAT_OK;  // every response is empty
   CutConst c;
@@ -463,11 +508,11 @@ int nat_select_cutlaw(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const
   NAT_LAUNCH_CHECK("cutlaw_sum_kernel");
   cutlaw_scan_kernel<<<1, 1024, 0, stream>>>(chunk_off, n_chunks);
   NAT_LAUNCH_CHECK("cutlaw_scan_kernel");
-  cutlaw_starts_kernel<<<n_chunks, kSelThreads, 0, stream>>>(B, cu_seqlens, n_tot, q, chunk_off,
-                                                             rstart);
+  cutlaw_starts_kernel<<<n_chunks, kSelThreads, 0, stream>>>(c, B, cu_seqlens, n_tot, q, chunk_off,
+                                                             rstart, udraw);
   NAT_LAUNCH_CHECK("cutlaw_starts_kernel");
-  cutlaw_final_kernel<<<n_chunks, kSelThreads, 0, stream>>>(c, B, cu_seqlens, n_tot, q, chunk_off,
-                                                            rstart, mask, pi, cut_len);
+  cutlaw_final_kernel<<<n_chunks, kSelThreads, 0, stream>>>(B, cu_seqlens, n_tot, q, chunk_off,
+                                                            rstart, udraw, mask, pi, cut_len);
   NAT_LAUNCH_CHECK("cutlaw_final_kernel");
   return NAT_OK;
 }

@@ -301,6 +301,12 @@ def test_cut_law_selection(lengths):
         q[7] = 0.0                      # a zero mass inside a response
         q[11] = -1.0                    # negative and NaN count as zero
         q[13] = np.nan
+        q[15] = 2.0                     # masses of 1 and above saturate at 2^32 - 1
+        q[16] = 1.0
+        q[17] = 1e-40                   # subnormal: below the fixed-point quantum
+        q[18] = np.float32(2.0 ** -33)  # just below one quantum, and exactly one
+        q[19] = np.float32(2.0 ** -32)
+        q[20] = np.inf
         q[cu[2]:cu[3]] = 0.0            # a response whose law has no mass at all: kept whole
     if B > 7:
         q[cu[7]:cu[8]] = 1.0 / 64       # dyadic uniform law

@@ -373,6 +373,8 @@ def test_cutlaw_survival_is_the_suffix_sum_of_q():
     mask, pi, cut = select_cutlaw(cu, q, seed=1)
     k = cutlaw_counts(q)
     assert np.array_equal(k, np.floor(q.astype(np.float64) * 2.0 ** 32).astype(np.uint64))
+    assert list(cutlaw_counts(np.array([1.0, 2.5, 0.5, -1.0, np.nan], dtype=np.float32))) == \
+        [2 ** 32 - 1, 2 ** 32 - 1, 2 ** 31, 0, 0]
     for i, Ti in enumerate(T):
         if Ti == 0:
             assert cut[i] == 0
