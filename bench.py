@@ -79,6 +79,25 @@ def dram_traffic(kind, d, V, chunk_rows):
     return None, "shape not covered by the capture"
 
 
+def dh_k_parts(chunk_rows, d, V, slots=74):
+    """K parts the library uses for the dHidden contraction of one row chunk on a whole B200
+    (74 CTA pairs): the smallest count up to 8 that fills the pairs' rounds to 95 %.  Only
+    used to count this script's own kernel launches."""
+    tiles = (chunk_rows // 512) * ((d + 255) // 256)
+    kb = (V + 63) // 64
+    best, best_eff = 1, 0.0
+    for parts in range(1, 9):
+        if parts > 1 and kb // parts < 64:
+            break
+        units = tiles * parts
+        eff = units / (-(-units // slots) * slots) if units else 0.0
+        if eff > best_eff + 1e-9:
+            best, best_eff = parts, eff
+        if eff >= 0.95:
+            return parts
+    return best
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -482,13 +501,16 @@ def run_ours(args, w):
     chunk_rows = min(cap_pad, 8192)
     n_chunks = (cap_pad + chunk_rows - 1) // chunk_rows
     sel_launches = 1 + (1 if w.sel_mode == "urs" else 2) + (3 if w.sel_mode == "urs" else 2)
+    k_parts = dh_k_parts(chunk_rows, w.d, w.V)
     if w.dtype == "f32":
         launches = sel_launches + 2 + 3
     elif args.route == "single":
-        # gather, references; per chunk 9; tail: fallback note, 5 one-hot kernels, loss sum
-        launches = sel_launches + 2 + 9 * n_chunks + 7
+        # gather, row references; per chunk kE, finalize, kDh (+ its finalize when the K range
+        # is cut into parts), kDw and the predicated redo (kFwd, finalize, kDz, kDh (+), kDw);
+        # tail: fallback note, five kernels of the ordered one-hot pass, loss sum
+        launches = sel_launches + 2 + (9 + (2 if k_parts > 1 else 0)) * n_chunks + 7
     else:
-        launches = sel_launches + 3 + (2 + 3 * n_chunks + 5)
+        launches = sel_launches + 4 + 2 + (3 + (1 if k_parts > 1 else 0)) * n_chunks + 5
     kernel = ("nat_tc_kernel<kE|kDh|kDw> (the launches inside nat_policy_loss_fwd_bwd)"
               if args.route == "single" else
               "nat_tc_kernel<kFwd|kDz|kDh|kDw> (nat_policy_loss_fwd + nat_policy_loss_bwd)")
