@@ -232,12 +232,16 @@ select_kernel(SelConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
     if (inside) {
       const int T = (int)(end - start);
       const int t_first = (int)(n0 - start) + 1;
+      // the kept tokens are the first L - t_first + 1 of the thread's 16 (clamped)
+      const int keep = min(max(L - t_first + 1, 0), kTokPerThread);
+      bits = (1u << keep) - 1u;
+      // numerators T - t + 1 by exact float subtraction (integers below 2^24): one
+      // int-to-float conversion per thread instead of one per token
+      const float a0 = (float)(T - t_first + 1);
+      const int ones = C - t_first + 1;  // tokens of the thread with t <= C
 #pragma unroll
-      for (int j = 0; j < kTokPerThread; ++j) {
-        const int t = t_first + j;
-        bits |= (t <= L ? 1u : 0u) << j;
-        pr[j] = (t <= C) ? 1.f : div_rn_by((float)(T - t + 1), den, rden);
-      }
+      for (int j = 0; j < kTokPerThread; ++j)
+        pr[j] = (j < ones) ? 1.f : div_rn_by(a0 - (float)j, den, rden);
       *reinterpret_cast<uint4*>(mask + n0) = bits_to_bytes(bits);
     } else {
       alignas(16) uint8_t m[kTokPerThread];

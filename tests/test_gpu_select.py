@@ -336,3 +336,48 @@ def test_cut_law_selection(lengths):
     assert np.array_equal(st.sel_idx[:n].cpu().numpy(), si)
     assert np.array_equal(st.sel_resp[:n].cpu().numpy(), sr)
     assert np.array_equal(st.sel_offsets[:B + 1].cpu().numpy(), so)
+
+
+# ------------------------------------------------------------ maximum sizes
+@pytest.mark.parametrize("mode", ["urs", "rpc"])
+def test_stream_close_to_the_int32_limit(mode):
+    """n_tot = 65535 responses of 32767 tokens = 2,147,385,345 (< 2^31): the largest packed
+    stream the int32 indices can address.  The oracle evaluates a sample of responses on
+    their own (their draws depend only on the global response index); the lists are checked
+    in full against plain torch reductions of the mask and on sampled segments."""
+    B, T = 65535, 32767
+    n_tot = B * T
+    assert n_tot < 2 ** 31 and n_tot > 2 ** 31 - 2 ** 17
+    cu = torch.arange(0, n_tot + 1, T, dtype=torch.int64, device="cuda").to(torch.int32)
+    st = NatStep(B // 5, 5, 64, 512, torch.float32, n_tot, want_grads=False)
+    kw = dict(p=0.5, min_cut=100, seed=21, offset=(1 << 33) + 5)
+    st.select(cu, mode, **kw)
+    st.compact(cu)
+    torch.cuda.synchronize()
+    n_sel = int(st.n_sel.item())
+    per_resp = st.mask[:n_tot].view(B, T).sum(dim=1, dtype=torch.int64)
+    assert n_sel == int(per_resp.sum().item())
+    offs = torch.zeros(B + 1, dtype=torch.int64, device="cuda")
+    offs[1:] = per_resp.cumsum(0)
+    assert torch.equal(st.sel_offsets.to(torch.int64), offs)
+    rng = np.random.default_rng(3)
+    one = wl.cu_from_lengths(np.array([T], dtype=np.int32))
+    for i in [0, 1, B - 1, B - 2] + [int(x) for x in rng.integers(2, B - 2, size=4)]:
+        m, p, c = oracle.select(MODE_ID[mode], one, resp_base=i, **kw)
+        lo = i * T
+        assert np.array_equal(st.mask[lo:lo + T].cpu().numpy(), m), i
+        assert np.array_equal(st.pi[lo:lo + T].cpu().numpy().view(np.uint32), p.view(np.uint32)), i
+        if c is not None:
+            assert int(st.cut_len[i].item()) == int(c[0])
+        k0, k1 = int(offs[i].item()), int(offs[i + 1].item())
+        want = torch.nonzero(st.mask[lo:lo + T]).flatten() + lo
+        assert torch.equal(st.sel_idx[k0:k1].to(torch.int64), want), i
+        assert bool((st.sel_resp[k0:k1] == i).all()), i
+    if mode == "rpc":
+        # the generic compaction of the same mask gives the same lists
+        idx_prefix = st.sel_idx[:n_sel].clone()
+        st.sel_idx.fill_(-1)
+        st.compact(cu, from_mask=True)
+        torch.cuda.synchronize()
+        assert int(st.n_sel.item()) == n_sel
+        assert torch.equal(st.sel_idx[:n_sel], idx_prefix)
