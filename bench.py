@@ -871,6 +871,9 @@ def main():
                     help="N > 1: the ranks split ONE batch by prompt groups (global batch size in "
                          "the weights, global response index in the selection) and all-reduce "
                          "loss and dW every step; strong scaling")
+    ap.add_argument("--spawn", action="store_true",
+                    help="start the ranks through the launcher even for --gpus 1 (checks the "
+                         "launcher itself on a single-GPU machine)")
     ap.add_argument("--allreduce-dw", action="store_true",
                     help="N > 1, independent batches: also sum loss and dW over the ranks inside "
                          "every step (timing of the exchange only)")
@@ -888,8 +891,9 @@ def main():
     if args.mode == "source-hash":
         print(kernel_source_hash())
         return
-    if args.impl == "ours" and args.mode == "step" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
-        sys.exit(launch_ranks(args, sys.argv[1:]))
+    if (args.impl == "ours" and args.mode == "step" and (args.gpus > 1 or args.spawn) and
+            "WORLD_SIZE" not in os.environ):
+        sys.exit(launch_ranks(args, [a for a in sys.argv[1:] if a != "--spawn"]))
     w = pick_workload(args)
     if args.impl == "reference":
         run_reference(args, w)

@@ -26,12 +26,13 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
   constexpr uint32_t kWeylA = 0x9E3779B9u, kWeylB = 0xBB67AE85u;
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hiA = __umulhi(kMulA, c0), loA = kMulA * c0;
-    const uint32_t hiB = __umulhi(kMulB, c2), loB = kMulB * c2;
-    c0 = hiB ^ c1 ^ k0;
-    c1 = loB;
-    c2 = hiA ^ c3 ^ k1;
-    c3 = loA;
+    // each 32x32->64 product as one wide multiply (its halves are the round's hi and lo)
+    const unsigned long long pA = (unsigned long long)kMulA * c0;
+    const unsigned long long pB = (unsigned long long)kMulB * c2;
+    c0 = (uint32_t)(pB >> 32) ^ c1 ^ k0;
+    c1 = (uint32_t)pB;
+    c2 = (uint32_t)(pA >> 32) ^ c3 ^ k1;
+    c3 = (uint32_t)pA;
     k0 += kWeylA;
     k1 += kWeylB;
   }
