@@ -49,6 +49,16 @@ def test_mid_bf16_multi_chunk_shapes():
     parity.run_case(w, seed=3)
 
 
+def test_k_parts_with_ragged_columns_and_vocabulary():
+    # V large enough for the dHidden contraction to run in K parts (their partial tiles meet
+    # in the float32 scratch), with d not a multiple of the 256-column block and V not a
+    # multiple of the 64-entry k-block: the last column block and the last k-block are ragged
+    w = wl.variant(wl.WORKLOADS["mid"], d=320, V=20001, P=4, G=8, len_lo=60, len_hi=200, p=0.75,
+                   old_noise=0.3)
+    parity.run_case(w, seed=3, routes=(False, True))
+    parity.run_case(wl.variant(w, d=64, V=9000, w_scale=0.5), seed=4, routes=(False, True))
+
+
 def test_twin_0p6b():
     parity.run_case(wl.WORKLOADS["twin_0p6b"], seed=0, routes=(False, True))
 
