@@ -55,12 +55,18 @@ def load_peaks():
 
 
 def kernel_source_hash():
-    """sha256 over the sources of the tensor-core loss kernels: the ncu counters kept under
-    profiles/ carry the hash of the sources they were taken from."""
+    """sha256 over the code of the tensor-core loss kernels (comments and blank lines
+    left out): the ncu counters kept under profiles/ carry the hash of the code they
+    were taken from."""
     h = hashlib.sha256()
     for name in KERNEL_SOURCES:
-        with open(os.path.join(ROOT, "paper_2603_06619_b200", "csrc", name), "rb") as f:
-            h.update(f.read())
+        with open(os.path.join(ROOT, "paper_2603_06619_b200", "csrc", name)) as f:
+            text = f.read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        for line in text.splitlines():
+            line = re.sub(r"//.*", "", line).strip()
+            if line:
+                h.update(line.encode() + b"\n")
     return h.hexdigest()[:16]
 
 

@@ -8,7 +8,10 @@
 //                                        stay in tensor memory and registers.
 //   kDz   S = Hc W^T  recomputed         epilogue: -g exp(S - lse) -> bf16 into
 //                                        the bounded scratch dZ[chunk, V].
-//   kDh   dH = dZ W   (rows x d, K = V)  epilogue: + g W[y] (one-hot term) -> bf16.
+//   kDh   dH = dZ W   (rows x d, K = V)  epilogue: + g W[y] (one-hot term) -> bf16; or, with
+//                                        the K range cut into parts so that the work units
+//                                        fill the device, an fp32 reduction of each part
+//                                        into a scratch from which a small pass forms dH.
 //   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 reduction into dW (TMA reduce-add).
 //   kE    S = Hc W^T  single-pass variant  epilogue: E = exp(S - mref) -> bf16 into the
 //                                        same scratch, row sums of E, target pick.
@@ -29,7 +32,9 @@
 // overlaps the next tile's MMAs.  kE / kDh / kDw: two sub-tiles per CTA (512x256 per CTA
 // pair, a quarter less operand traffic); their accumulators fill tensor memory, the
 // epilogue is exposed and therefore leaves through a shared-memory staging block by TMA
-// store (kE) or TMA reduction (kDw) instead of scattered 16-byte accesses.
+// store (kE) or TMA reduction (kDw, kDh in K parts) instead of scattered 16-byte accesses.
+// Work units are taken round-robin by the CTA pairs; kE's units are single vocabulary
+// tiles ordered so that the pairs sweep the vocabulary together (see decode_unit).
 // Every mbarrier wait is bounded; a wait that runs out raises the block's
 // abort flag and NAT_DEV_TIMEOUT in the workspace's status word.
 #include <cuda_bf16.h>
