@@ -381,3 +381,22 @@ def test_stream_close_to_the_int32_limit(mode):
         torch.cuda.synchronize()
         assert int(st.n_sel.item()) == n_sel
         assert torch.equal(st.sel_idx[:n_sel], idx_prefix)
+
+
+def test_prefix_compaction_clamps_cut_lengths():
+    # cut lengths outside [0, T_i] (a caller's mistake) are clamped, never used as they are
+    T = np.array([5, 0, 9, 3], dtype=np.int32)
+    cu = wl.cu_from_lengths(T)
+    n_tot = int(cu[-1])
+    cut = torch.tensor([7, 4, -2, 3], dtype=torch.int32, device="cuda")      # -> 5, 0, 0, 3
+    st = NatStep(1, 4, 64, 512, torch.float32, n_tot, want_grads=False)
+    for t in (st.sel_idx, st.sel_resp):
+        t.fill_(-9)
+    nat.nat_compact_prefix(4, torch.from_numpy(cu).cuda(), n_tot, cut, st.sel_idx, st.sel_resp,
+                           st.sel_offsets, st.n_sel, st.cap)
+    torch.cuda.synchronize()
+    assert int(st.n_sel.item()) == 8
+    assert st.sel_offsets.cpu().tolist() == [0, 5, 5, 5, 8]
+    assert st.sel_idx[:8].cpu().tolist() == [0, 1, 2, 3, 4, 14, 15, 16]
+    assert st.sel_resp[:8].cpu().tolist() == [0] * 5 + [3] * 3
+    assert int(st.sel_idx[8:].max()) == -9
