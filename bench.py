@@ -309,7 +309,7 @@ def run_ours(args, w):
     if world > 1:
         dist.barrier()
 
-    sharded = args.sharded and world > 1
+    sharded = args.sharded          # with one rank: the same path, the exchange a no-op
     exchange_on = sharded or (args.allreduce_dw and world > 1)
     if sharded:
         # ONE batch, split by prompt groups: this rank holds responses [lo, hi) of it, keeps
@@ -557,7 +557,8 @@ def run_ours(args, w):
     line = {
         "metric": METRIC, "value": n_all / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms,
-        "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
+        "higher_is_better": True, "scaling": "strong" if sharded and world > 1 else "weak",
+        "vs_baseline": None,
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": w.name, "P": w.P, "G": w.G, "d": w.d, "V": w.V,
                    "selection": w.sel_mode, "p": w.p, "min_cut": w.min_cut, "beta": w.beta,
