@@ -439,3 +439,72 @@ def test_cutlaw_draw_boundaries_and_frequencies():
     freq = np.bincount(cuts, minlength=5)[1:] / R
     z = (freq - q) / np.sqrt(q * (1 - q) / R)
     assert np.abs(z).max() < 4.5
+
+
+# ---------------------------------------------- draws: ranges, ends and strictness
+def test_rpc_cut_reaches_both_ends_with_the_uniform_frequency():
+    """L_i is uniform on {C..T}: both ends are attained and every value has frequency
+    1/(T - C + 1) (z-test over 8000 responses, fixed seed).  A cut law that never reaches T
+    would leave the last token with inclusion probability 0 < p_{i,T}."""
+    T, C, R = 7, 3, 8000
+    _, pi, cuts = select(SEL_RPC, _cu([T] * R), min_cut=C, seed=17)
+    n = T - C + 1
+    freq = np.bincount(cuts, minlength=T + 1)[C:] / R
+    assert cuts.min() == C and cuts.max() == T
+    z = (freq - 1.0 / n) / math.sqrt((1.0 / n) * (1 - 1.0 / n) / R)
+    assert np.abs(z).max() < 4.5
+    # and the realised frequency of keeping token t is pi_t
+    kept = (np.arange(1, T + 1)[None, :] <= cuts[:, None]).mean(0)
+    p = pi[:T].astype(np.float64)
+    zz = (kept - p) / np.sqrt(np.maximum(p * (1 - p), 1e-12) / R)
+    assert np.abs(zz[C:]).max() < 4.5 and np.all(kept[:C] == 1.0)
+
+
+def test_survival_draw_is_24_bit_and_the_comparison_strict():
+    """Each response's schedule is built from its own draw, recomputed here from the
+    generator: with p_2 = k 2^-24 (k the 24-bit draw itself) the token is NOT kept
+    (u < p fails at equality), with p_2 = (k + 1) 2^-24 it is.  A coarser draw, or a
+    non-strict comparison, flips one of the two."""
+    from oracle.philox import philox4x32_10 as ph
+    B = 64
+    x0 = ph(0, np.arange(B), 2, 0, 5, 0)[0]
+    k = (x0 >> np.uint64(8)).astype(np.int64)
+    assert (k % 2 == 1).sum() > 10 and (k % 2 == 0).sum() > 10      # both parities occur
+    cu = _cu([2] * B)
+    at = np.stack([np.ones(B), k * 2.0 ** -24], axis=1).astype(np.float32).ravel()
+    above = np.stack([np.ones(B), (k + 1) * 2.0 ** -24], axis=1).astype(np.float32).ravel()
+    ok = k > 0                                                       # a schedule must stay positive
+    at[1::2][~ok] = 2.0 ** -24
+    _, cut_at = select_survival(cu, at, seed=5)
+    _, cut_above = select_survival(cu, above, seed=5)
+    assert np.all(cut_at[ok] == 1) and np.all(cut_above == 2)
+
+
+def test_cutlaw_unit_counts_make_every_cut_equally_likely():
+    """Masses of one fixed-point quantum each (q = 2^-32): S = (T, .., 2, 1) and r is uniform
+    on {0..T-1}, so L = T - r takes every value in {1..T} with probability 1/T; a non-strict
+    comparison S_t >= r would never produce L = 1."""
+    T, R = 4, 6000
+    q = np.full(T * R, 2.0 ** -32, dtype=np.float32)
+    mask, pi, cuts = select_cutlaw(_cu([T] * R), q, seed=23)
+    assert np.array_equal(pi[:T], np.array([1.0, 0.75, 0.5, 0.25], dtype=np.float32))
+    freq = np.bincount(cuts, minlength=T + 1)[1:] / R
+    assert cuts.min() == 1 and cuts.max() == T
+    z = (freq - 0.25) / math.sqrt(0.25 * 0.75 / R)
+    assert np.abs(z).max() < 4.5
+
+
+def test_rpc_draw_layout_is_the_documented_one():
+    """The cut of response i comes from words 0 and 1 of the Philox block with counter
+    (0, i, 1, offset_lo): u = x1 2^32 + x0 (the layout the C header documents and the CUDA
+    kernels follow).  T - C + 1 = 2^40-scale ranges do not exist, so the high word decides L:
+    using x0 twice, or the words swapped, changes the cuts."""
+    from oracle.philox import philox4x32_10 as ph
+    T, C = 32768, 1
+    for seed in range(40):
+        x0, x1, _, _ = ph(0, 3, 1, 9, seed, 0)
+        u = (int(x1) << 32) | int(x0)
+        want = C + ((u * (T - C + 1)) >> 64)
+        _, _, cut = select(SEL_RPC, _cu([T]), min_cut=C, seed=seed, offset=9, resp_base=3)
+        assert cut[0] == want
+        assert want == C + ((int(x1) * (T - C + 1)) >> 32)      # the high word alone fixes L here
