@@ -34,10 +34,15 @@ ROW_BLOCK = 8192
 
 
 def _sample_rows(n, rng, k_random=40):
+    """Selected rows the oracle evaluates: stream ends, tile and chunk edges, random rows, and
+    one random row of every 8192-row chunk (a chunk that was skipped, repeated or misplaced
+    cannot hide between the samples)."""
     edges = [0, 1, 127, 128, 129, 255, 256, 511, 512, 8191, 8192, 8193, 16383, 16384, n - 129,
              n - 128, n - 2, n - 1]
     rows = {r for r in edges if 0 <= r < n}
     rows |= set(int(x) for x in rng.integers(0, n, size=k_random))
+    for lo in range(0, n, ROW_BLOCK):
+        rows.add(int(rng.integers(lo, min(lo + ROW_BLOCK, n))))
     return np.array(sorted(rows), dtype=np.int64)
 
 
