@@ -159,6 +159,29 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def board_gemm_rate(seconds=3.0, n=8192):
+    """Sustained bf16 rate of the library's plain GEMM (torch.matmul, n^3) on THIS board, now:
+    looped for `seconds` under the power cap, second half timed.  The boards of a pool settle
+    at different clocks under the same cap, so this puts a same-board figure beside the
+    pool-wide measured peak.  The library is called for this denominator only."""
+    import torch
+    a = torch.randn(n, n, device="cuda").to(torch.bfloat16)
+    b = torch.randn(n, n, device="cuda").to(torch.bfloat16)
+    c = torch.empty(n, n, device="cuda", dtype=torch.bfloat16)
+    ms = _time(lambda: torch.matmul(a, b, out=c), 4, warmup=2)
+    reps = max(8, int(seconds * 1e3 / ms))
+    for _ in range(reps // 2):
+        torch.matmul(a, b, out=c)
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    ms = _time(lambda: torch.matmul(a, b, out=c), reps - reps // 2, warmup=0)
+    clk = sampler.stop()
+    return {"tflops": 2.0 * n ** 3 / (ms * 1e-3) / 1e12, "sm_mhz": clk.get("sm_mhz"),
+            "power_w": clk.get("power_w"),
+            "how": f"torch.matmul {n}^3 bf16 looped for about {seconds:.0f} s after the timed "
+                   "region, second half timed"}
+
+
 def host_cores():
     try:
         return len(os.sched_getaffinity(0))
@@ -608,6 +631,11 @@ def run_ours(args, w):
         line["nccl"] = nccl_log_summary()
     if args.route == "two":
         line["fwd_ms"], line["bwd_ms"] = first_ms, loss_call_ms - first_ms
+    if not args.no_cpu_baseline and world == 1 and w.dtype == "bf16":
+        # the same fraction against what the library's GEMM sustains on this very board
+        lib = board_gemm_rate()
+        line["roofline"]["library_gemm_this_board"] = lib
+        line["roofline"]["frac_of_this_board"] = call_tflops / lib["tflops"]
     if not args.no_cpu_baseline and world == 1:
         rate, secs, n, _ = oracle_sample_rate(w, seed=0, rows=args.ref_rows)
         line["cpu_baseline"] = {
