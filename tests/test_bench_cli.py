@@ -66,3 +66,16 @@ def test_sharded_batches_partition_the_global_batch_and_share_W():
     assert torch.equal(shards[0]["W"], shards[1]["W"])                      # replicated head
     assert not torch.equal(shards[0]["hidden"][:8], shards[1]["hidden"][:8])
     assert sum(b["n_tot"] for b in shards) == int(T_all.sum())
+
+
+def test_a_bad_clock_record_is_measured_again():
+    ok = {"sm_mhz": 1300.0, "sm_max_mhz": 1965.0, "reasons": ["sw_power_cap"], "samples": 40}
+    assert not bench.clocks_rejected(ok)                                     # power cap: kept
+    assert bench.clocks_rejected(dict(ok, reasons=["hw_thermal_slowdown", "sw_power_cap"]))
+    assert bench.clocks_rejected(dict(ok, reasons=["sw_thermal_slowdown"]))
+    assert bench.clocks_rejected(dict(ok, reasons=["hw_slowdown"]))
+    assert bench.clocks_rejected(dict(ok, sm_mhz=900.0, reasons=[]))         # a leftover lock
+    assert not bench.clocks_rejected(dict(ok, sm_mhz=1900.0, reasons=[]))
+    assert not bench.clocks_rejected(dict(ok, sm_mhz=900.0, reasons=[], samples=1))  # too short
+    assert not bench.clocks_rejected(None)
+    assert not bench.clocks_rejected({"sm_mhz": None, "reasons": ["nvidia-smi unavailable"]})
