@@ -120,6 +120,36 @@ def check_loss(st, ref_sel, nb, w, backward=True, hidden_is_compact=False, clip=
     return out, ref
 
 
+def settle_clip_decisions(batch, nb, ref_sel, clip=(0.2, 0.2), band=2e-3, shift=2e-2):
+    """Move tokens off the clip bounds, in the inputs of both sides.
+
+    The derivative of the clipped surrogate (Eq. grpo-surrogate) jumps where the ratio
+    crosses 1 - clip_lo or 1 + clip_hi, so a token whose ratio lies within the forward's
+    numerical error of a bound has no unique gradient: the kernels' forward (bf16 products,
+    fp32 sums) and the fp64 oracle may land on different sides, and both are right.  Tokens
+    with |log r - log bound| < band * max(1, max lse / 16) (r from the oracle's logp) get
+    their old_logp moved by ten times that, away from the bound.  Returns how many moved."""
+    fwd = oracle.policy_loss_fwd(nb["hidden"], nb["W"], nb["targets"], nb["old_logp"],
+                                 ref_sel["adv"], ref_sel["pi"], nb["cu_seqlens"],
+                                 ref_sel["sel_idx"], ref_sel["sel_resp"], clip_lo=clip[0],
+                                 clip_hi=clip[1])
+    si = np.asarray(ref_sel["sel_idx"], dtype=np.int64)
+    mag = max(1.0, float(np.abs(fwd["lse"]).max(initial=0)) / 16.0)
+    old = nb["old_logp"]
+    logr = fwd["logp"] - old[si].astype(np.float64)
+    moved = 0
+    for bound in (np.log1p(clip[1]), np.log1p(-clip[0])):
+        near = np.abs(logr - bound) < band * mag
+        if near.any():
+            # log r = logp - old_logp: lower old_logp to push a ratio further above the bound
+            step = np.where(logr[near] >= bound, -1.0, 1.0) * (shift * mag)
+            old[si[near]] = (old[si[near]].astype(np.float64) + step).astype(np.float32)
+            moved += int(near.sum())
+    if moved:
+        batch["old_logp"].copy_(torch.from_numpy(old))
+    return moved
+
+
 def run_case(w, seed=0, offset=0, backward=True, device="cuda", fused=False, routes=None,
              **batch_kw):
     """One seeded batch through the library and the oracle.  ``routes`` lists the library
@@ -128,6 +158,8 @@ def run_case(w, seed=0, offset=0, backward=True, device="cuda", fused=False, rou
     batch = wl.make_batch(w, seed=seed, device=device, **batch_kw)
     nb = wl.to_numpy(batch)
     ref_sel = oracle_selection(w, nb, seed, offset)
+    if backward:
+        settle_clip_decisions(batch, nb, ref_sel)
     out, ref = None, None
     for f in ([fused] if routes is None else routes):
         st = gpu_step(w, batch, seed, offset, backward=backward, fused=f)
