@@ -10,8 +10,9 @@
 //                                        the bounded scratch dZ[chunk, V].
 //   kDh   dH = dZ W   (rows x d, K = V)  epilogue: + g W[y] (one-hot term) -> bf16; or, with
 //                                        the K range cut into parts so that the work units
-//                                        fill the device, an fp32 reduction of each part
-//                                        into a scratch from which a small pass forms dH.
+//                                        fill the device, each part's fp32 partial tile
+//                                        stored into its slice of a scratch whose slices a
+//                                        small pass adds in part order to form dH.
 //   kDw   dW += dZ^T Hc (V x d, K = rows) epilogue: fp32 reduction into dW (TMA reduce-add).
 //   kE    S = Hc W^T  single-pass variant  epilogue: E = exp(S - mref) -> bf16 into the
 //                                        same scratch, row sums of E, target pick.
@@ -32,7 +33,7 @@
 // overlaps the next tile's MMAs.  kE / kDh / kDw: two sub-tiles per CTA (512x256 per CTA
 // pair, a quarter less operand traffic); their accumulators fill tensor memory, the
 // epilogue is exposed and therefore leaves through a shared-memory staging block by TMA
-// store (kE) or TMA reduction (kDw, kDh in K parts) instead of scattered 16-byte accesses.
+// store (kE, kDh in K parts) or TMA reduction (kDw) instead of scattered 16-byte accesses.
 // Work units are taken round-robin by the CTA pairs; kE's units are single vocabulary
 // tiles ordered so that the pairs sweep the vocabulary together (see decode_unit).
 // Every mbarrier wait is bounded; a wait that runs out raises the block's
@@ -105,7 +106,7 @@ struct Unit {
   int mb;      // block along the accumulator's M dimension
   int nt_lo;   // first and one-past-last block along N
   int nt_hi;
-  int sp;      // vocabulary split (kFwd, kDz, kE)
+  int sp;      // vocabulary split (kFwd, kDz, kE) or K part (kDh)
   int kb_lo;   // k-blocks of this unit: the whole K range, or one of k_splits parts of it (kDh)
   int kb_hi;
 };
@@ -175,10 +176,10 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Shape& s, i
     // (K part, row block, column block), the column block varying fastest: the pairs in
     // flight work on one K part, i.e. on the same half of W and the same few slabs of the
     // numerators (measured 2 % faster per step than taking the parts of a tile in turn)
-    w.sp = 0;
     const int per_ks = s.mblocks * s.nblocks;
     const int ks = u / per_ks;
     const int rem = u - ks * per_ks;
+    w.sp = ks;  // the K part: its partial tile has a slice of the scratch to itself
     w.mb = rem / s.nblocks;
     w.nt_lo = rem - w.mb * s.nblocks;
     w.nt_hi = w.nt_lo + 1;
@@ -642,8 +643,9 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
                 *reinterpret_cast<uint4*>(dst + 8 * g8) = make_uint4(
                     packed[4 * g8], packed[4 * g8 + 1], packed[4 * g8 + 2], packed[4 * g8 + 3]);
           } else if (MODE == kDh && SUBS == 2 && p.k_splits > 1) {
-            // partial tile of a K part: added into the float32 scratch through the warp's
-            // staging block (TMA reduction), like kDw below; rows past the chunk are clipped
+            // partial tile of a K part: stored into the part's own slice of the float32
+            // scratch through the warp's staging block (a TMA store of whole lines); the
+            // slices are added in part order by dh_finalize_kernel, so the sum's order is fixed
             uint8_t* stage = staging + (warp - 2) * 4096;
             if (lane == 0) tc::bulk_wait_read_all();
             __syncwarp();
@@ -654,7 +656,7 @@ nat_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ 
             tc::fence_proxy_async();
             __syncwarp();
             if (lane == 0) {
-              tc::tma_reduce_add_2d(&mapC, stage, col0, lrow);
+              tc::tma_store_2d(&mapC, stage, col0, w.sp * p.chunk_rows + lrow);
               tc::bulk_commit();
             }
           } else if (MODE == kDh) {
@@ -877,15 +879,17 @@ fused_finalize_kernel(TokenCtx c, const int32_t* __restrict__ n_sel, int cap, in
   }
 }
 
-// dHidden of one row chunk from the float32 sums of the K parts (kDh with k_splits > 1):
-//   dH[k, :] = scale_k * acc[k - row0, :] + g_k W[y_k, :]   (one block per row).
+// dHidden of one row chunk from the float32 partial tiles of the K parts (kDh with
+// k_splits > 1), slice p of `acc` holding part p's [chunk_rows, d] partial sums:
+//   dH[k, :] = scale_k * (sum over parts in ascending order of acc[p][k - row0, :]) + g_k W[y_k, :]
+// (one block per row).
 __global__ void __launch_bounds__(128)
 dh_finalize_kernel(const float* __restrict__ acc, const float* __restrict__ row_scale,
                    const float* __restrict__ g, const __nv_bfloat16* __restrict__ W,
                    const int32_t* __restrict__ targets, const int32_t* __restrict__ sel_idx,
                    const int32_t* __restrict__ n_sel, int cap, int row0, int chunk_rows, int d,
-                   int V, __nv_bfloat16* __restrict__ dH, const int32_t* __restrict__ flag,
-                   int run_if) {
+                   int V, int parts, __nv_bfloat16* __restrict__ dH,
+                   const int32_t* __restrict__ flag, int run_if) {
   if (predicate_off(flag, run_if)) return;
   int n = *n_sel;
   n = n < cap ? n : cap;
@@ -900,8 +904,14 @@ dh_finalize_kernel(const float* __restrict__ acc, const float* __restrict__ row_
     const float4* a = reinterpret_cast<const float4*>(acc + (size_t)r * d);
     const uint4* wsrc = reinterpret_cast<const uint4*>(W + (size_t)y * d);
     uint4* dst = reinterpret_cast<uint4*>(dH + (size_t)k * d);
+    const size_t slice4 = (size_t)chunk_rows * d / 4;  // float4 elements per part
     for (int j = threadIdx.x; j < vec; j += blockDim.x) {
-      const float4 a0 = a[2 * j], a1 = a[2 * j + 1];
+      float4 a0 = a[2 * j], a1 = a[2 * j + 1];
+      for (int q = 1; q < parts; ++q) {
+        const float4 b0 = a[q * slice4 + 2 * j], b1 = a[q * slice4 + 2 * j + 1];
+        a0.x += b0.x; a0.y += b0.y; a0.z += b0.z; a0.w += b0.w;
+        a1.x += b1.x; a1.y += b1.y; a1.z += b1.z; a1.w += b1.w;
+      }
       const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
       const uint4 wv = __ldg(wsrc + j);
       const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
@@ -1087,7 +1097,8 @@ int pair_slots();
 // Number of K parts of the dHidden contraction.  Its work units are (512-row block,
 // 256-column block) tiles over the whole vocabulary as K: few and long (256 for a full chunk
 // at d = 4096), so the last round of the CTA pairs is mostly empty.  Cutting K into parts
-// multiplies the units; the parts of a tile meet in a float32 scratch.  The smallest count
+// multiplies the units; every part has its own float32 slice of a scratch and a small pass
+// adds the slices in part order (a fixed order: dHidden is reproducible).  The smallest count
 // that fills the rounds to 95 % is taken (1 when CTA pairs are not available).
 int pick_k_splits(int tiles, int kb, int slots) {
   if (slots <= 0 || tiles <= 0) return 1;
@@ -1144,7 +1155,7 @@ Layout make_layout(const nat_loss_params& p, int64_t cap) {
   off = align_up(off, 1024);
   L.off_hc = take(sizeof(__nv_bfloat16) * (size_t)L.cap_pad * p.d);
   L.off_hs = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * p.d);
-  L.off_dhacc = take(L.dh_splits > 1 ? sizeof(float) * (size_t)L.chunk_rows * p.d : 0);
+  L.off_dhacc = take(L.dh_splits > 1 ? sizeof(float) * (size_t)L.dh_splits * L.chunk_rows * p.d : 0);
   L.off_dz = take(sizeof(__nv_bfloat16) * (size_t)L.chunk_rows * L.ldz);
   L.total = off;
   return L;
@@ -1438,7 +1449,7 @@ struct Maps {
   CUtensorMap hcK, wK, wK2, dzK, wMn, dzMn, hcMn, hsMn;  // wK2: 128-row boxes for CTA pairs
   CUtensorMap dzSt;  // the numerator scratch as a store target: 64 columns x 32 rows
   CUtensorMap dwRed;  // dW as a reduction target (valid only when the call has a dW)
-  CUtensorMap dhAcc;  // the float32 scratch of the dHidden K parts as a reduction target
+  CUtensorMap dhAcc;  // the float32 scratch of the dHidden K parts: [parts x chunk_rows, d]
 };
 
 int encode_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
@@ -1456,7 +1467,8 @@ int encode_maps(const LossArgs& a, const Layout& L, const Ws& w, Maps* m) {
   m->dwRed = m->dzSt;
   if (a.dW != nullptr && (s = make_map_f32(&m->dwRed, a.dW, a.p.d, a.p.V)) != NAT_OK) return s;
   m->dhAcc = m->dzSt;
-  if (L.dh_splits > 1 && (s = make_map_f32(&m->dhAcc, w.dhacc, a.p.d, L.chunk_rows)) != NAT_OK)
+  if (L.dh_splits > 1 &&
+      (s = make_map_f32(&m->dhAcc, w.dhacc, a.p.d, (uint64_t)L.dh_splits * L.chunk_rows)) != NAT_OK)
     return s;
   return NAT_OK;
 }
@@ -1519,15 +1531,13 @@ int launch_dh(const LossArgs& a, const Layout& L, const Ws& w, const Maps& m, Tc
   p.run_if = run_if;
   const bool parts = L.dh_splits > 1 && pair_slots() > 0;
   p.k_splits = parts ? L.dh_splits : 1;
-  if (parts)
-    NAT_CUDA(cudaMemsetAsync(w.dhacc, 0, sizeof(float) * (size_t)L.chunk_rows * a.p.d, a.stream));
   if ((s = launch_tc<kDh>(m.dzK, m.wMn, m.wMn, parts ? m.dhAcc : m.hcK, p, mb, nb_d * p.k_splits,
                           a.stream)) != NAT_OK)
     return s;
   if (parts) {
     dh_finalize_kernel<<<L.chunk_rows < 4096 ? L.chunk_rows : 4096, 128, 0, a.stream>>>(
         w.dhacc, p.row_scale, w.g, reinterpret_cast<const __nv_bfloat16*>(a.W), a.targets,
-        a.sel_idx, a.n_sel, (int)a.cap, p.row0, L.chunk_rows, a.p.d, a.p.V,
+        a.sel_idx, a.n_sel, (int)a.cap, p.row0, L.chunk_rows, a.p.d, a.p.V, p.k_splits,
         reinterpret_cast<__nv_bfloat16*>(a.dHidden), flag, run_if);
     NAT_LAUNCH_CHECK("dh_finalize_kernel");
   }

@@ -312,6 +312,21 @@ def test_dW_is_reproducible_when_many_tokens_share_a_target():
             assert torch.equal(dW1, st.dW)
 
 
+def test_dHidden_is_reproducible_when_the_vocabulary_is_cut_into_many_K_parts():
+    # d = 1024 with few row blocks: the dHidden contraction runs in eight K parts, whose
+    # partial tiles must be added in the same order on every run
+    w = wl.variant(wl.WORKLOADS["twin_0p6b"], P=2, len_lo=200, len_hi=400, p=1.0)
+    batch = wl.make_batch(w, seed=5, device="cuda")
+    for fused in (False, True):
+        st = parity.gpu_step(w, batch, 5, 0, fused=fused)
+        dH1, dW1, loss1 = st.dH.clone(), st.dW.clone(), st.loss.clone()
+        for _ in range(4):
+            st.run(batch, w.sel_mode, p=w.p, seed=5, fused=fused)
+            torch.cuda.synchronize()
+            assert torch.equal(dH1, st.dH) and torch.equal(dW1, st.dW)
+            assert torch.equal(loss1, st.loss)
+
+
 def test_target_outside_the_vocabulary_is_reported_and_left_out():
     w = wl.WORKLOADS["mid"]
     batch = wl.make_batch(w, seed=0, device="cuda")
