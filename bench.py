@@ -251,8 +251,12 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    rows = args.ref_rows
-    rate, _, n, times = oracle_sample_rate(w, seed=0, rows=rows, repeats=max(1, args.steps))
+    # W warm-up passes and K timed ones; the per-step sample shrinks with K + W so that the
+    # whole run stays within a few minutes (the rate is linear in the rows)
+    passes = max(1, args.steps) + max(0, args.warmup)
+    rows = args.ref_rows if passes <= 8 else max(96, args.ref_rows * 8 // passes)
+    rate, _, n, times = oracle_sample_rate(w, seed=0, rows=rows, repeats=passes)
+    times = times[max(0, args.warmup):]
     ms = 1e3 * statistics.mean(times)
     cores = host_cores()
     sample = f"{n} selected rows of the {w.name} head per step (fp64 loss fwd+bwd, all of V)"
