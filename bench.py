@@ -251,10 +251,11 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    # W warm-up passes and K timed ones; the per-step sample shrinks with K + W so that the
-    # whole run stays within a few minutes (the rate is linear in the rows)
+    # W warm-up passes and K timed ones over the same bounded sample (its size is kept: the
+    # oracle's per-call setup, widening W_lm to fp64, would weigh more on a smaller one);
+    # about 8 s per pass on 16 cores at the default sample, so K = 20 ends within a few minutes
     passes = max(1, args.steps) + max(0, args.warmup)
-    rows = args.ref_rows if passes <= 8 else max(96, args.ref_rows * 8 // passes)
+    rows = args.ref_rows
     rate, _, n, times = oracle_sample_rate(w, seed=0, rows=rows, repeats=passes)
     times = times[max(0, args.warmup):]
     ms = 1e3 * statistics.mean(times)
