@@ -127,17 +127,19 @@ prefix_write_kernel(int B, const int32_t* __restrict__ cu, const int32_t* __rest
 // ------------------------------------------------------------- cut laws
 // Fixed-point mass of one token: min(floor(q 2^32), 2^32 - 1) for q > 0, else 0 (NaN and
 // negative masses count as 0).  Taken from the float's bits with integer operations only
-// (a float-to-integer conversion instruction runs at a sixteenth of their rate): q = m 2^e
-// with the 24-bit significand m, so floor(q 2^32) is m shifted by e + 32.
+// (a float-to-integer conversion instruction runs at a sixteenth of their rate): for
+// 0 < q < 1, q = m 2^(e - 150) with the 24-bit significand m, so floor(q 2^32) is
+// (m 2^8) >> (126 - e), a 32-bit value shifted right; the shift instruction yields 0 for
+// amounts of 32 and more, which covers the tiny masses (subnormals included, whose missing
+// hidden bit no longer matters there).
 __device__ __forceinline__ uint32_t cutlaw_count(float q) {
   const uint32_t bits = __float_as_uint(q);
-  if (!(q > 0.f)) return 0u;                       // zero, negative, NaN
-  const int exp = (int)(bits >> 23);               // sign bit is clear here
-  if (exp >= 127) return 0xFFFFFFFFu;              // q >= 1 (infinity included)
-  if (exp == 0) return 0u;                         // subnormal: below 2^-126
-  const uint32_t m = (bits & 0x7FFFFFu) | 0x800000u;
-  const int sh = exp - 118;                        // (exp - 150) + 32; at most 8 here
-  return sh >= 0 ? m << sh : (sh > -24 ? m >> -sh : 0u);
+  const uint32_t e = bits >> 23;                   // biased exponent where q > 0
+  const uint32_t m8 = (bits << 8) | 0x80000000u;   // significand with its hidden bit, times 2^8
+  uint32_t r;
+  asm("shr.u32 %0, %1, %2;" : "=r"(r) : "r"(m8), "r"(126u - e));  // amounts >= 32 give 0
+  if (e >= 127u) r = 0xFFFFFFFFu;                  // q >= 1 (infinity included)
+  return q > 0.f ? r : 0u;                         // zero, negative, NaN
 }
 
 __device__ __forceinline__ void load_counts(const float* __restrict__ q, int64_t n0, int64_t n_tot,
