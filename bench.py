@@ -795,7 +795,7 @@ def select_compact_stress(log2_tokens=28, T=8192, reps=5):
     ms = _time(lambda: nat.nat_select_cutlaw(B, cu, n_tot, q, 1, 0, st.mask, st.pi, st.cut_len, ws),
                reps)
     row("nat_select_cutlaw (random law)", "-", ms,
-        "4 B/token read (the law) + 5 B/token written; executed: the law is read 3 times", 9.0 * n_tot)
+        "4 B/token read (the law) + 5 B/token written; executed: the law is read twice", 9.0 * n_tot)
     del q
     st.grpo_adv(torch.zeros(B, device="cuda"))
     ms = _time(lambda: st.grpo_adv(torch.zeros(B, device="cuda")), reps)

@@ -3,10 +3,10 @@
 // suffix sum of the law (a scan over the packed stream).
 //
 // Both are bound by HBM traffic.  nat_compact_prefix writes 8 bytes per selected token and
-// reads only the B cut lengths.  nat_select_cutlaw reads the law three times (4 bytes per
-// token each: chunk sums, prefix at the response starts, final pass) and writes mask and pi
-// (5 bytes per token); all sums are exact 64-bit integers of fixed-point masses, so the
-// result does not depend on how the scan is split over chunks and threads.
+// reads only the B cut lengths.  nat_select_cutlaw reads the law twice (4 bytes per token
+// each: chunk sums with the local prefixes at the response starts, final pass) and writes
+// mask and pi (5 bytes per token); all sums are exact 64-bit integers of fixed-point
+// masses, so the result does not depend on how the scan is split over chunks and threads.
 #include <cstdint>
 
 #include "nat_common.cuh"
@@ -184,22 +184,54 @@ __device__ __forceinline__ unsigned long long block_excl_scan(unsigned long long
   return before + incl - v;
 }
 
-// Pass 1: the sum of the counts of each 4096-token chunk.
+// Pass 1: the sum of the counts of each 4096-token chunk and, for every response that starts
+// strictly inside the chunk, the sum of the chunk's counts before its first token (the
+// chunk's counts are kept in shared memory so that a start in the middle of a thread's 16
+// tokens can be resolved).  A start on a chunk boundary needs no such local part.
 __global__ void __launch_bounds__(kSelThreads)
-cutlaw_sum_kernel(const float* __restrict__ q, int64_t n_tot,
-                  unsigned long long* __restrict__ chunk_sum) {
+cutlaw_sum_kernel(int B, const int32_t* __restrict__ cu, const float* __restrict__ q,
+                  int64_t n_tot, unsigned long long* __restrict__ chunk_sum,
+                  unsigned long long* __restrict__ rlocal) {
   __shared__ unsigned long long warp_tot[kSelThreads / 32];
-  const int64_t n0 = (int64_t)blockIdx.x * kSelBlockTokens + (int64_t)threadIdx.x * kTokPerThread;
+  __shared__ unsigned long long thread_excl[kSelThreads];
+  __shared__ uint32_t k_s[kSelThreads * kPiPad];  // 17 slots per thread: no bank conflicts
+  __shared__ int first_s;
+  const int64_t chunk0 = (int64_t)blockIdx.x * kSelBlockTokens;
+  const int64_t chunk_lim = chunk0 + (int64_t)kSelBlockTokens;  // starts inside: (chunk0, chunk_lim)
+  if (threadIdx.x < 32) {  // first response whose start is > chunk0
+    int w0, first_in = 0;
+    const int64_t v = cu_window(cu, B, chunk0, n_tot, &w0);
+    if (!window_first(__ballot_sync(0xFFFFFFFFu, v > chunk0), w0, &first_in))
+      first_in = warp_upper_bound(cu, B, chunk0, 0);
+    if (threadIdx.x == 0) first_s = first_in;
+  }
+  const int64_t n0 = chunk0 + (int64_t)threadIdx.x * kTokPerThread;
   uint32_t k[kTokPerThread];
   unsigned long long s = 0;
-  if (n0 < n_tot) {
-    load_counts(q, n0, n_tot, k);
 #pragma unroll
-    for (int j = 0; j < kTokPerThread; ++j) s += k[j];
-  }
+  for (int j = 0; j < kTokPerThread; ++j) k[j] = 0;
+  if (n0 < n_tot) load_counts(q, n0, n_tot, k);
+#pragma unroll
+  for (int j = 0; j < kTokPerThread; ++j) s += k[j];
   unsigned long long total;
-  block_excl_scan(s, warp_tot, &total);
+  const unsigned long long excl = block_excl_scan(s, warp_tot, &total);  // has a __syncthreads
   if (threadIdx.x == 0) chunk_sum[blockIdx.x] = total;
+  const int first_in = first_s;
+  // block-uniform: no response starts strictly inside this chunk
+  if (first_in > B || (int64_t)cu[first_in] >= chunk_lim) return;
+  thread_excl[threadIdx.x] = excl;
+#pragma unroll
+  for (int j = 0; j < kTokPerThread; ++j) k_s[threadIdx.x * kPiPad + j] = k[j];
+  __syncthreads();
+  for (int i = first_in + (int)threadIdx.x; i <= B; i += kSelThreads) {
+    const int64_t n = cu[i];
+    if (n >= chunk_lim) break;
+    const int rel = (int)(n - chunk0);  // 1 .. 4095; counts past the stream's end are zero
+    const int t = rel / kTokPerThread, j = rel % kTokPerThread;
+    unsigned long long g = thread_excl[t];
+    for (int e = 0; e < j; ++e) g += k_s[t * kPiPad + e];
+    rlocal[i] = g;
+  }
 }
 
 // Pass 2: exclusive scan of the chunk sums in place by one block; total to chunk_sum[n_chunks].
@@ -239,79 +271,37 @@ struct CutConst {
   uint32_t k0, k1, off_lo, resp_base;
 };
 
-// Pass 3: G[cu_i], the sum of all counts before the first token of response i, for every
-// response whose start lies in this chunk (the last chunk also takes the starts equal to
-// n_tot), and the response's 64-bit draw.  The chunk's counts are kept in shared memory so
-// that a start in the middle of a thread's 16 tokens can be resolved.
-__global__ void __launch_bounds__(kSelThreads)
-cutlaw_starts_kernel(CutConst c, int B, const int32_t* __restrict__ cu, int64_t n_tot,
-                     const float* __restrict__ q, const unsigned long long* __restrict__ chunk_off,
+// Pass 3: G[cu_i], the sum of all counts before the first token of response i: the scanned
+// sum of the chunks before the one that holds cu_i plus the local part of pass 1 (none when
+// cu_i sits on a chunk boundary; chunk_off has one entry past the last chunk, the grand
+// total, for starts at the stream's end), and the response's 64-bit draw.  One thread per
+// response.
+__global__ void __launch_bounds__(256)
+cutlaw_starts_kernel(CutConst c, int B, const int32_t* __restrict__ cu,
+                     const unsigned long long* __restrict__ chunk_off,
                      unsigned long long* __restrict__ rstart,
                      unsigned long long* __restrict__ udraw) {
-  __shared__ unsigned long long warp_tot[kSelThreads / 32];
-  __shared__ unsigned long long thread_excl[kSelThreads];
-  __shared__ uint32_t k_s[kSelThreads * kPiPad];  // 17 slots per thread: no bank conflicts
-  __shared__ int first_s;
-  const int64_t chunk0 = (int64_t)blockIdx.x * kSelBlockTokens;
-  const int64_t chunk_end = min(chunk0 + (int64_t)kSelBlockTokens, n_tot);
-  if (threadIdx.x < 32) {  // first response whose start is >= chunk0
-    int w0, first_in = 0;
-    const int64_t v = cu_window(cu, B, chunk0, n_tot, &w0);
-    if (!window_first(__ballot_sync(0xFFFFFFFFu, v >= chunk0), w0, &first_in))
-      first_in = warp_upper_bound(cu, B, chunk0 - 1, 0);
-    if (threadIdx.x == 0) first_s = first_in;
-  }
-  __syncthreads();
-  const int first_in = first_s;
-  // nothing starts here: cu[first_in] is past the chunk (block-uniform, so all threads leave)
-  const bool last = (chunk_end == n_tot);
-  if (first_in > B) return;
-  {
-    const int64_t c0 = cu[first_in];
-    if (c0 > chunk_end || (c0 == chunk_end && !last)) return;
-  }
-  const int64_t n0 = chunk0 + (int64_t)threadIdx.x * kTokPerThread;
-  uint32_t k[kTokPerThread];
-  unsigned long long s = 0;
-#pragma unroll
-  for (int j = 0; j < kTokPerThread; ++j) k[j] = 0;
-  if (n0 < n_tot) load_counts(q, n0, n_tot, k);
-#pragma unroll
-  for (int j = 0; j < kTokPerThread; ++j) {
-    s += k[j];
-    k_s[threadIdx.x * kPiPad + j] = k[j];
-  }
-  unsigned long long total;
-  const unsigned long long excl = block_excl_scan(s, warp_tot, &total);
-  thread_excl[threadIdx.x] = excl;
-  __syncthreads();
-  const unsigned long long base = chunk_off[blockIdx.x];
-  for (int i = first_in + (int)threadIdx.x; i <= B; i += kSelThreads) {
-    const int64_t n = cu[i];
-    if (n > chunk_end || (n == chunk_end && !last)) break;
-    if (i < B) {
-      const Philox4 x = philox4x32_10(0u, c.resp_base + (uint32_t)i, 3u, c.off_lo, c.k0, c.k1);
-      udraw[i] = ((unsigned long long)x.y << 32) | (unsigned long long)x.x;
-    }
-    if (n == chunk_end) {  // the stream's end (only in the last chunk)
-      rstart[i] = base + total;
-    } else {
-      const int rel = (int)(n - chunk0);
-      const int t = rel / kTokPerThread, j = rel % kTokPerThread;
-      unsigned long long g = base + thread_excl[t];
-      for (int e = 0; e < j; ++e) g += k_s[t * kPiPad + e];
-      rstart[i] = g;
-    }
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i > B) return;
+  const int64_t n = cu[i];
+  const unsigned long long local = (n % kSelBlockTokens) != 0 ? rstart[i] : 0ull;
+  rstart[i] = chunk_off[n / kSelBlockTokens] + local;
+  if (i < B) {
+    const Philox4 x = philox4x32_10(0u, c.resp_base + (uint32_t)i, 3u, c.off_lo, c.k0, c.k1);
+    udraw[i] = ((unsigned long long)x.y << 32) | (unsigned long long)x.x;
   }
 }
 
 // double(x), correctly rounded.  Below 2^52 the value is exact and comes from one integer
 // OR and one addition (2^52 + x has x in its low significand bits); the conversion
 // instruction, which is slow, is left to the counts that large.
+__device__ __forceinline__ double below_2p52_to_double(unsigned long long x) {
+  return __dadd_rn(__longlong_as_double((long long)(0x4330000000000000ull | x)),
+                   -4503599627370496.0);
+}
+
 __device__ __forceinline__ double u64_to_double(unsigned long long x) {
-  if (x < (1ull << 52))
-    return __dadd_rn(__longlong_as_double((long long)(0x4330000000000000ull | x)),
-                     -4503599627370496.0);
+  if (x < (1ull << 52)) return below_2p52_to_double(x);
   return __ull2double_rn(x);
 }
 
@@ -373,12 +363,22 @@ cutlaw_final_kernel(int B, const int32_t* __restrict__ cu, int64_t n_tot,
     uint32_t bits = 0;
     float* pr = pi_s + threadIdx.x * kPiPad;
     if (cnt == kTokPerThread && n0 + kTokPerThread <= end && S1 != 0ull) {
-      // the usual case: the thread's 16 tokens lie inside one response whose law has mass
+      // the usual case: the thread's 16 tokens lie inside one response whose law has mass;
+      // every survival count is at most S1, so one test picks the conversion for all of them
+      if (S1 < (1ull << 52)) {
 #pragma unroll
-      for (int j = 0; j < kTokPerThread; ++j) {
-        bits |= (St > r ? 1u : 0u) << j;
-        pr[j] = __double2float_rn(__dmul_rn(u64_to_double(St), inv_total));
-        St -= k[j];
+        for (int j = 0; j < kTokPerThread; ++j) {
+          bits |= (St > r ? 1u : 0u) << j;
+          pr[j] = __double2float_rn(__dmul_rn(below_2p52_to_double(St), inv_total));
+          St -= k[j];
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < kTokPerThread; ++j) {
+          bits |= (St > r ? 1u : 0u) << j;
+          pr[j] = __double2float_rn(__dmul_rn(u64_to_double(St), inv_total));
+          St -= k[j];
+        }
       }
       // the kept tokens are a prefix of the response; this thread holds its last one when
       // some but not all of its tokens are kept, or all are and the next token (St is its
@@ -506,12 +506,13 @@ int nat_select_cutlaw(int32_t B, const int32_t* cu_seqlens, int64_t n_tot, const
   c.k1 = (uint32_t)((seed >> 32) ^ (offset >> 32));
   c.off_lo = (uint32_t)(offset & 0xFFFFFFFFull);
   c.resp_base = (uint32_t)resp_base;
-  cutlaw_sum_kernel<<<n_chunks, kSelThreads, 0, stream>>>(q, n_tot, chunk_off);
+  cutlaw_sum_kernel<<<n_chunks, kSelThreads, 0, stream>>>(B, cu_seqlens, q, n_tot, chunk_off,
+                                                          rstart);
   NAT_LAUNCH_CHECK("cutlaw_sum_kernel");
   cutlaw_scan_kernel<<<1, 1024, 0, stream>>>(chunk_off, n_chunks);
   NAT_LAUNCH_CHECK("cutlaw_scan_kernel");
-  cutlaw_starts_kernel<<<n_chunks, kSelThreads, 0, stream>>>(c, B, cu_seqlens, n_tot, q, chunk_off,
-                                                             rstart, udraw);
+  cutlaw_starts_kernel<<<(B + 256) / 256, 256, 0, stream>>>(c, B, cu_seqlens, chunk_off, rstart,
+                                                            udraw);
   NAT_LAUNCH_CHECK("cutlaw_starts_kernel");
   cutlaw_final_kernel<<<n_chunks, kSelThreads, 0, stream>>>(B, cu_seqlens, n_tot, q, chunk_off,
                                                             rstart, udraw, mask, pi, cut_len);
