@@ -93,9 +93,12 @@ __device__ __forceinline__ float div_rn_by(float a, float b, float rcp_b) {
   return __fmaf_rn(r, rcp_b, q0);
 }
 
+// Bit w set iff word w of the block lies below the threshold (1 .. 2^32; at 2^32 every
+// word does: the test is the same for all threads, and below it the compares are 32-bit).
 __device__ __forceinline__ uint32_t philox_below(const Philox4& r, uint64_t thr) {
-  return ((uint64_t)r.x < thr ? 1u : 0u) | ((uint64_t)r.y < thr ? 2u : 0u) |
-         ((uint64_t)r.z < thr ? 4u : 0u) | ((uint64_t)r.w < thr ? 8u : 0u);
+  if ((thr >> 32) != 0ull) return 0xFu;
+  const uint32_t t = (uint32_t)thr;
+  return (r.x < t ? 1u : 0u) | (r.y < t ? 2u : 0u) | (r.z < t ? 4u : 0u) | (r.w < t ? 8u : 0u);
 }
 
 __global__ void __launch_bounds__(kSelThreads)
